@@ -1,0 +1,219 @@
+/*
+ * spiffy.h -- C ABI of libspiffy: the verification hot path of Spiffy
+ * (speculative decoding for masked-diffusion LLMs with directed draft graphs),
+ * written for NVIDIA B200 (sm_100a).
+ *
+ * One verification step scores N draft states of one L-token block in a single
+ * packed forward pass of the target model and then decides how far the block
+ * may advance.  This library holds the two model-independent, data-parallel
+ * pieces of that step:
+ *
+ *   spiffy_graph_attention   the packed attention of Sec. 4.3 (mask of Fig. 3):
+ *                            every draft state attends to the cached context
+ *                            and, bidirectionally, to its own block only;
+ *   spiffy_unmask_decide     steps 1-4 of Algorithm 1 (the function Next() of
+ *                            App. A) evaluated for every node of the graph;
+ *   spiffy_accept_walk       step 5 of Algorithm 1: the walk through the draft
+ *                            graph (Sec. 4.4.1, Eqs. draft-graph-1..3) to the
+ *                            deepest accepted node.
+ *
+ * Vocabulary (paper notation in brackets where it differs):
+ *   B  batch of independent sequences            N  nodes of the draft graph,
+ *   L  block length [L]                             node 0 = the true block
+ *   P  cached context length (keys/values of X')    X_k(t), nodes 1..N-1 = the
+ *   Hq, Hkv  query / key-value heads                draft blocks [D = N-1]
+ *   d  head dimension                            V  vocabulary size [V]
+ *   tau  confidence threshold of dynamic unmasking; S  static unmasking rate
+ *
+ * Conventions common to every entry point
+ *   - Every data pointer is a DEVICE pointer owned by the caller; the library
+ *     neither allocates nor frees device memory.  Descriptors are plain host
+ *     structs, read before the call returns.
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*,
+ *     NULL = the default stream) and never synchronise the device.
+ *   - Scratch memory is caller-provided: size it with the *_workspace() query.
+ *     Its contents on entry are arbitrary; calls sharing one workspace must be
+ *     ordered on one stream.
+ *   - Tensor base addresses must be 16-byte aligned, else SPIFFY_EINVAL.
+ *   - Host-detectable problems return a status code and launch nothing.
+ *     Device-detectable problems set bits in a caller-provided status word and
+ *     yield a defined output; no kernel traps, asserts or waits unboundedly.
+ *   - Thread-safe for calls on distinct streams with distinct workspaces.
+ */
+#ifndef SPIFFY_H_
+#define SPIFFY_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SPIFFY_OK = 0,
+  SPIFFY_EINVAL = 1,       /* null pointer, bad size, misaligned tensor */
+  SPIFFY_EUNSUPPORTED = 2, /* shape or dtype outside the stated limits */
+  SPIFFY_EWORKSPACE = 3,   /* workspace missing or too small */
+  SPIFFY_EGRAPH = 4,       /* reserved for host-side graph validation */
+  SPIFFY_ECUDA = 5         /* a CUDA runtime call failed (launch error) */
+} spiffy_status;
+
+typedef enum { SPIFFY_F32 = 0, SPIFFY_BF16 = 1 } spiffy_dtype;
+
+/* Unmasking rule of step 3 of Algorithm 1.
+ * TOPS:      the S most confident still-masked positions (Sec. 3.1, S_t = S).
+ * THRESHOLD: every still-masked position whose confidence is > tau (strict,
+ *            Sec. 3.1 "threshold-based dynamic unmasking"); when none passes,
+ *            the single most confident one, so that decoding always advances. */
+typedef enum { SPIFFY_RULE_TOPS = 0, SPIFFY_RULE_THRESHOLD = 1 } spiffy_rule;
+
+/* Bits of the device status words. */
+#define SPIFFY_DEV_NONFINITE 1 /* a logits row held NaN/+inf or only -inf     */
+#define SPIFFY_DEV_BADGRAPH 2  /* parent list malformed (offsets or indices)   */
+#define SPIFFY_DEV_TIMEOUT 4   /* a bounded on-chip wait gave up               */
+
+/* Attention kernel selection (spiffy_attn_desc.kernel). */
+#define SPIFFY_ATTN_AUTO 0   /* tensor-core kernel when the shape allows it   */
+#define SPIFFY_ATTN_SIMT 1   /* fp32 CUDA-core kernel (any supported shape)   */
+#define SPIFFY_ATTN_TCGEN05 2 /* tcgen05/TMEM kernel or SPIFFY_EUNSUPPORTED   */
+
+/* ------------------------------------------------------------------------- */
+/* Packed draft-graph attention (Sec. 4.3; mask semantics: caption of Fig. 3) */
+/* ------------------------------------------------------------------------- */
+typedef struct {
+  int32_t batch;      /* B >= 1                                              */
+  int32_t n_nodes;    /* N >= 1                                              */
+  int32_t block_len;  /* L in [1, 64]                                        */
+  int32_t prefix_len; /* P >= 0 context keys shared by all nodes             */
+  int32_t n_q_heads;  /* Hq                                                  */
+  int32_t n_kv_heads; /* Hkv, divides Hq; query head h reads kv head
+                         h / (Hq/Hkv)                                        */
+  int32_t head_dim;   /* d in {64, 128}                                      */
+  int32_t dtype;      /* spiffy_dtype of q, k, v and out                     */
+  float scale;        /* softmax scale; 0 means 1/sqrt(d)                    */
+  int32_t kernel;     /* SPIFFY_ATTN_*                                       */
+} spiffy_attn_desc;
+
+/* Bytes of scratch spiffy_graph_attention needs for this shape (may be 0). */
+size_t spiffy_graph_attention_workspace(const spiffy_attn_desc* desc);
+
+/*
+ * out[b,n,l,h,:] = sum_j softmax_j(scale * <q[b,n,l,h,:], k_j>) * v_j, where j
+ * runs over the P context keys of sequence b and the L keys of node n's OWN
+ * block -- no other node's block, the root's included.  Attention inside the
+ * block is bidirectional.  Positional encoding is the caller's: q and k arrive
+ * already rotated, every node using the true block's positions (Sec. 4.3).
+ *
+ * Layouts (row-major, innermost last), all of dtype desc->dtype:
+ *   q, out             [B][N][L][Hq][d]
+ *   k_prefix, v_prefix [B][P][Hkv][d]     (may be NULL when P == 0)
+ *   k_block, v_block   [B][N][L][Hkv][d]
+ * dev_status: one int32 on the device, OR-ed with SPIFFY_DEV_* bits; may be
+ * NULL.  Accumulation is fp32; the result is rounded once to desc->dtype.
+ */
+spiffy_status spiffy_graph_attention(const spiffy_attn_desc* desc,
+                                     const void* q, const void* k_prefix,
+                                     const void* v_prefix, const void* k_block,
+                                     const void* v_block, void* out,
+                                     int32_t* dev_status, void* workspace,
+                                     size_t workspace_bytes, void* cuda_stream);
+
+/* ------------------------------------------------------------------------- */
+/* Decision: steps 1-4 of Algorithm 1 for every node (Next() of App. A)      */
+/* ------------------------------------------------------------------------- */
+typedef struct {
+  int32_t batch;         /* B                                                */
+  int32_t n_nodes;       /* N                                                */
+  int32_t block_len;     /* L in [1, 64]                                     */
+  int32_t vocab;         /* V >= 1                                           */
+  int32_t logits_dtype;  /* spiffy_dtype                                     */
+  int64_t row_stride;    /* elements between consecutive logits rows, >= V;
+                            row_stride * sizeof(element) must be a multiple
+                            of 16                                            */
+  int32_t mask_token_id; /* token id that marks a still-masked position      */
+  int32_t rule;          /* spiffy_rule                                      */
+  int32_t top_s;         /* S of RULE_TOPS (>= 1); ignored by THRESHOLD      */
+  float threshold;       /* tau of RULE_THRESHOLD                            */
+} spiffy_decide_desc;
+
+size_t spiffy_unmask_decide_workspace(const spiffy_decide_desc* desc);
+
+/*
+ * For every node (b,n) and every position l with block_tokens[b,n,l] ==
+ * mask_token_id, reduce the V logits of row (b,n,l) to
+ *   top_tok = argmax_v x_v (lowest v on ties),
+ *   conf    = max_v softmax(x)_v = 1 / sum_v exp(x_v - max x)
+ * (steps 1-2), then choose the set U of positions to unmask by desc->rule
+ * (step 3; ties in confidence go to the lower position).  Step 4, the next
+ * state, is state with top_tok written at the positions of U; it is returned
+ * implicitly as (top_tok, unmask_bits).
+ *
+ *   logits       [B][N][L] rows of V elements, desc->row_stride apart; rows of
+ *                already-unmasked positions are never read
+ *   block_tokens [B][N][L] int32, the state of every node
+ *   conf         [B][N][L] fp32; -inf at unmasked positions
+ *   top_tok      [B][N][L] int32; the existing token at unmasked positions
+ *   unmask_bits  [B][N] uint64, bit l set when l is in U
+ *   n_unmask     [B][N] int32, |U| (0 for a node with nothing left to unmask)
+ *   dev_status   [B] int32, OR-ed with SPIFFY_DEV_NONFINITE when a row that was
+ *                read is not finite (its conf/top_tok are then unspecified);
+ *                may be NULL
+ * Math is fp32 on exactly up-converted inputs; the argmax compares input
+ * values, never probabilities.
+ */
+spiffy_status spiffy_unmask_decide(const spiffy_decide_desc* desc,
+                                   const void* logits,
+                                   const int32_t* block_tokens, float* conf,
+                                   int32_t* top_tok, uint64_t* unmask_bits,
+                                   int32_t* n_unmask, int32_t* dev_status,
+                                   void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream);
+
+/* ------------------------------------------------------------------------- */
+/* Acceptance: step 5 of Algorithm 1 over the draft graph of Sec. 4.4.1      */
+/* ------------------------------------------------------------------------- */
+/*
+ * Per sequence b: cur = 0 (the true block).  Repeat: let next(cur) be
+ * state(cur) with top_tok written at unmask_bits(cur).  Among the nodes m that
+ * list cur as a parent, in ascending m, take the first whose state equals
+ * next(cur) on all L tokens; if there is one it is accepted (its distribution
+ * replaces the target's), cur = m; otherwise stop.  A node with an empty
+ * unmask set ends the walk.
+ *
+ *   parent_off [B][N+1] int32, CSR offsets into parent_idx, relative to the
+ *              start of sequence b's own slice: the slice of sequence b begins
+ *              at parent_idx + b * parent_cap
+ *   parent_idx [B][parent_cap] int32, parents of node m at
+ *              [parent_off[b][m], parent_off[b][m+1]); a parent index must be
+ *              smaller than its child's (topological order), node 0 has none
+ *   accepted_node [B] deepest accepted node (0 = no draft accepted)
+ *   n_accepted    [B] number of accepted drafts = hops taken; the block has
+ *                 advanced n_accepted + 1 denoising steps on one model call
+ *   path          [B][N] visited nodes, root first, padded with -1
+ *   next_block    [B][L] next(accepted_node): the new true block
+ *   dev_status    [B] OR-ed with SPIFFY_DEV_BADGRAPH when an offset or index is
+ *                 out of range (such entries are ignored); may be NULL
+ * Uses desc->batch, n_nodes, block_len only.
+ */
+spiffy_status spiffy_accept_walk(const spiffy_decide_desc* desc,
+                                 const int32_t* block_tokens,
+                                 const int32_t* parent_off,
+                                 const int32_t* parent_idx, int32_t parent_cap,
+                                 const int32_t* top_tok,
+                                 const uint64_t* unmask_bits,
+                                 int32_t* accepted_node, int32_t* n_accepted,
+                                 int32_t* path, int32_t* next_block,
+                                 int32_t* dev_status, void* cuda_stream);
+
+/* Static description of a status code; never NULL. */
+const char* spiffy_status_string(spiffy_status status);
+
+/* Launch counter: number of kernels this library has launched in this process
+ * since load (all entry points, all threads).  For benchmarks' bookkeeping. */
+uint64_t spiffy_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPIFFY_H_ */
