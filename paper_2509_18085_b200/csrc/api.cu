@@ -1,0 +1,150 @@
+// C ABI of libspiffy: argument validation and dispatch.  See include/spiffy.h
+// for the contract of every entry point.
+#include <atomic>
+
+#include "common.cuh"
+
+namespace spiffy {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+spiffy_status check_attn_desc(const spiffy_attn_desc* d) {
+  if (!d) return SPIFFY_EINVAL;
+  if (d->batch < 1 || d->n_nodes < 1 || d->block_len < 1 || d->prefix_len < 0 ||
+      d->n_q_heads < 1 || d->n_kv_heads < 1)
+    return SPIFFY_EINVAL;
+  if (d->n_q_heads % d->n_kv_heads != 0) return SPIFFY_EINVAL;
+  if (d->dtype != SPIFFY_F32 && d->dtype != SPIFFY_BF16) return SPIFFY_EINVAL;
+  if (!(d->scale >= 0.f) || !(d->scale < INFINITY)) return SPIFFY_EINVAL;
+  if (d->kernel < SPIFFY_ATTN_AUTO || d->kernel > SPIFFY_ATTN_TCGEN05) return SPIFFY_EINVAL;
+  if (d->block_len > 64) return SPIFFY_EUNSUPPORTED;
+  if (d->head_dim != 64 && d->head_dim != 128) return SPIFFY_EUNSUPPORTED;
+  if (d->n_nodes > 65535 || d->batch > 65535) return SPIFFY_EUNSUPPORTED;
+  return SPIFFY_OK;
+}
+
+bool use_tc(const spiffy_attn_desc& d) {
+  if (d.kernel == SPIFFY_ATTN_SIMT) return false;
+  return attention_tc_supported(d);
+}
+
+spiffy_status check_decide_desc(const spiffy_decide_desc* d, bool need_vocab) {
+  if (!d) return SPIFFY_EINVAL;
+  if (d->batch < 1 || d->n_nodes < 1 || d->block_len < 1) return SPIFFY_EINVAL;
+  if (d->block_len > 64) return SPIFFY_EUNSUPPORTED;
+  if ((int64_t)d->batch * d->n_nodes > 65535) return SPIFFY_EUNSUPPORTED;
+  if ((int64_t)d->batch * d->n_nodes * d->block_len > 65535) return SPIFFY_EUNSUPPORTED;
+  if (!need_vocab) return SPIFFY_OK;
+  if (d->vocab < 1) return SPIFFY_EINVAL;
+  if (d->logits_dtype != SPIFFY_F32 && d->logits_dtype != SPIFFY_BF16) return SPIFFY_EINVAL;
+  if (d->row_stride < d->vocab) return SPIFFY_EINVAL;
+  const int64_t esize = d->logits_dtype == SPIFFY_BF16 ? 2 : 4;
+  if ((d->row_stride * esize) % 16 != 0) return SPIFFY_EINVAL;
+  if (d->rule != SPIFFY_RULE_TOPS && d->rule != SPIFFY_RULE_THRESHOLD) return SPIFFY_EINVAL;
+  if (d->rule == SPIFFY_RULE_TOPS && d->top_s < 1) return SPIFFY_EINVAL;
+  if (d->rule == SPIFFY_RULE_THRESHOLD && !(d->threshold == d->threshold)) return SPIFFY_EINVAL;
+  return SPIFFY_OK;
+}
+
+}  // namespace
+}  // namespace spiffy
+
+using namespace spiffy;
+
+extern "C" {
+
+size_t spiffy_graph_attention_workspace(const spiffy_attn_desc* desc) {
+  if (check_attn_desc(desc) != SPIFFY_OK) return 0;
+  return use_tc(*desc) ? attention_tc_workspace_bytes(*desc) : 0;
+}
+
+spiffy_status spiffy_graph_attention(const spiffy_attn_desc* desc, const void* q,
+                                     const void* k_prefix, const void* v_prefix,
+                                     const void* k_block, const void* v_block,
+                                     void* out, int32_t* dev_status,
+                                     void* workspace, size_t workspace_bytes,
+                                     void* cuda_stream) {
+  const spiffy_status st = check_attn_desc(desc);
+  if (st != SPIFFY_OK) return st;
+  const spiffy_attn_desc d = *desc;
+  if (!q || !k_block || !v_block || !out) return SPIFFY_EINVAL;
+  if (d.prefix_len > 0 && (!k_prefix || !v_prefix)) return SPIFFY_EINVAL;
+  if (!aligned16(q) || !aligned16(k_block) || !aligned16(v_block) || !aligned16(out) ||
+      !aligned16(k_prefix) || !aligned16(v_prefix))
+    return SPIFFY_EINVAL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (use_tc(d)) {
+    const size_t need = attention_tc_workspace_bytes(d);
+    if (need > 0 && (!workspace || workspace_bytes < need || !aligned16(workspace)))
+      return SPIFFY_EWORKSPACE;
+    return launch_attention_tc(d, q, k_prefix, v_prefix, k_block, v_block, out,
+                               dev_status, workspace, stream);
+  }
+  if (d.kernel == SPIFFY_ATTN_TCGEN05) return SPIFFY_EUNSUPPORTED;
+  return launch_attention_simt(d, q, k_prefix, v_prefix, k_block, v_block, out, stream);
+}
+
+size_t spiffy_unmask_decide_workspace(const spiffy_decide_desc* desc) {
+  if (check_decide_desc(desc, true) != SPIFFY_OK) return 0;
+  return decide_workspace_bytes(*desc);
+}
+
+spiffy_status spiffy_unmask_decide(const spiffy_decide_desc* desc,
+                                   const void* logits,
+                                   const int32_t* block_tokens, float* conf,
+                                   int32_t* top_tok, uint64_t* unmask_bits,
+                                   int32_t* n_unmask, int32_t* dev_status,
+                                   void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream) {
+  const spiffy_status st = check_decide_desc(desc, true);
+  if (st != SPIFFY_OK) return st;
+  if (!logits || !block_tokens || !conf || !top_tok || !unmask_bits || !n_unmask)
+    return SPIFFY_EINVAL;
+  if (!aligned16(logits)) return SPIFFY_EINVAL;
+  const size_t need = decide_workspace_bytes(*desc);
+  if (!workspace || workspace_bytes < need || !aligned16(workspace)) return SPIFFY_EWORKSPACE;
+  return launch_decide(*desc, logits, block_tokens, conf, top_tok, unmask_bits,
+                       n_unmask, dev_status, workspace,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+spiffy_status spiffy_accept_walk(const spiffy_decide_desc* desc,
+                                 const int32_t* block_tokens,
+                                 const int32_t* parent_off,
+                                 const int32_t* parent_idx, int32_t parent_cap,
+                                 const int32_t* top_tok,
+                                 const uint64_t* unmask_bits,
+                                 int32_t* accepted_node, int32_t* n_accepted,
+                                 int32_t* path, int32_t* next_block,
+                                 int32_t* dev_status, void* cuda_stream) {
+  const spiffy_status st = check_decide_desc(desc, false);
+  if (st != SPIFFY_OK) return st;
+  if (!block_tokens || !parent_off || !parent_idx || !top_tok || !unmask_bits ||
+      !accepted_node || !n_accepted || !path || !next_block)
+    return SPIFFY_EINVAL;
+  if (parent_cap < 0) return SPIFFY_EINVAL;
+  return launch_walk(*desc, block_tokens, parent_off, parent_idx, parent_cap,
+                     top_tok, unmask_bits, accepted_node, n_accepted, path,
+                     next_block, dev_status, static_cast<cudaStream_t>(cuda_stream));
+}
+
+const char* spiffy_status_string(spiffy_status status) {
+  switch (status) {
+    case SPIFFY_OK: return "ok";
+    case SPIFFY_EINVAL: return "invalid argument (null, size, alignment)";
+    case SPIFFY_EUNSUPPORTED: return "shape or dtype outside the supported limits";
+    case SPIFFY_EWORKSPACE: return "workspace missing, misaligned or too small";
+    case SPIFFY_EGRAPH: return "malformed draft graph";
+    case SPIFFY_ECUDA: return "CUDA runtime error at launch";
+  }
+  return "unknown status";
+}
+
+uint64_t spiffy_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

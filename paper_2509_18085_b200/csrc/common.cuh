@@ -1,0 +1,53 @@
+// Internal helpers shared by the kernels of libspiffy (not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "spiffy.h"
+
+namespace spiffy {
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+// Every launch of the library goes through this counter (spiffy_launch_count).
+void count_launch(int n = 1);
+
+// Entry points implemented in the kernel files; all validated by the caller.
+spiffy_status launch_decide(const spiffy_decide_desc& d, const void* logits,
+                            const int32_t* block_tokens, float* conf,
+                            int32_t* top_tok, uint64_t* unmask_bits,
+                            int32_t* n_unmask, int32_t* dev_status, void* ws,
+                            cudaStream_t stream);
+size_t decide_workspace_bytes(const spiffy_decide_desc& d);
+int decide_splits(const spiffy_decide_desc& d, int64_t* chunk_elems);
+
+spiffy_status launch_walk(const spiffy_decide_desc& d,
+                          const int32_t* block_tokens,
+                          const int32_t* parent_off, const int32_t* parent_idx,
+                          int32_t parent_cap, const int32_t* top_tok,
+                          const uint64_t* unmask_bits, int32_t* accepted_node,
+                          int32_t* n_accepted, int32_t* path,
+                          int32_t* next_block, int32_t* dev_status,
+                          cudaStream_t stream);
+
+spiffy_status launch_attention_simt(const spiffy_attn_desc& d, const void* q,
+                                    const void* kp, const void* vp,
+                                    const void* kb, const void* vb, void* out,
+                                    cudaStream_t stream);
+
+// tcgen05 path: shape support query, workspace and launch.
+bool attention_tc_supported(const spiffy_attn_desc& d);
+size_t attention_tc_workspace_bytes(const spiffy_attn_desc& d);
+spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q,
+                                  const void* kp, const void* vp,
+                                  const void* kb, const void* vb, void* out,
+                                  int32_t* dev_status, void* ws,
+                                  cudaStream_t stream);
+
+inline spiffy_status check_launch() {
+  return cudaGetLastError() == cudaSuccess ? SPIFFY_OK : SPIFFY_ECUDA;
+}
+
+}  // namespace spiffy

@@ -1,0 +1,249 @@
+"""ctypes binding of ``libspiffy.so`` -- argument marshalling only.
+
+The three entry points carry the names of the C ABI (``include/spiffy.h``) and
+take torch CUDA tensors; every step of the path runs in the library's kernels.
+There is no CPU fallback: when the library has not been built, or a tensor is
+not on a CUDA device, the call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libspiffy.so")
+
+OK, EINVAL, EUNSUPPORTED, EWORKSPACE, EGRAPH, ECUDA = range(6)
+F32, BF16 = 0, 1
+RULE_TOPS, RULE_THRESHOLD = 0, 1
+DEV_NONFINITE, DEV_BADGRAPH, DEV_TIMEOUT = 1, 2, 4
+ATTN_AUTO, ATTN_SIMT, ATTN_TCGEN05 = 0, 1, 2
+
+EXPORTS = (
+    "spiffy_graph_attention_workspace", "spiffy_graph_attention",
+    "spiffy_unmask_decide_workspace", "spiffy_unmask_decide",
+    "spiffy_accept_walk", "spiffy_status_string", "spiffy_launch_count",
+)
+
+
+class SpiffyError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().spiffy_status_string(status).decode()
+        super().__init__(f"{where}: {msg} (status {status})")
+
+
+class AttnDesc(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("n_nodes", ctypes.c_int32),
+                ("block_len", ctypes.c_int32), ("prefix_len", ctypes.c_int32),
+                ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("scale", ctypes.c_float), ("kernel", ctypes.c_int32)]
+
+
+class DecideDesc(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("n_nodes", ctypes.c_int32),
+                ("block_len", ctypes.c_int32), ("vocab", ctypes.c_int32),
+                ("logits_dtype", ctypes.c_int32), ("row_stride", ctypes.c_int64),
+                ("mask_token_id", ctypes.c_int32), ("rule", ctypes.c_int32),
+                ("top_s", ctypes.c_int32), ("threshold", ctypes.c_float)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library; raises when it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with "
+                "`python -m paper_2509_18085_b200.build` (there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, sz, i32 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int32
+        L.spiffy_graph_attention_workspace.restype = sz
+        L.spiffy_graph_attention_workspace.argtypes = [ctypes.POINTER(AttnDesc)]
+        L.spiffy_graph_attention.restype = ctypes.c_int
+        L.spiffy_graph_attention.argtypes = [ctypes.POINTER(AttnDesc)] + [vp] * 8 + [sz, vp]
+        L.spiffy_unmask_decide_workspace.restype = sz
+        L.spiffy_unmask_decide_workspace.argtypes = [ctypes.POINTER(DecideDesc)]
+        L.spiffy_unmask_decide.restype = ctypes.c_int
+        L.spiffy_unmask_decide.argtypes = [ctypes.POINTER(DecideDesc)] + [vp] * 8 + [sz, vp]
+        L.spiffy_accept_walk.restype = ctypes.c_int
+        L.spiffy_accept_walk.argtypes = [ctypes.POINTER(DecideDesc), vp, vp, vp, i32] + [vp] * 8
+        L.spiffy_status_string.restype = ctypes.c_char_p
+        L.spiffy_status_string.argtypes = [ctypes.c_int]
+        L.spiffy_launch_count.restype = ctypes.c_uint64
+        L.spiffy_launch_count.argtypes = []
+        _lib = L
+    return _lib
+
+
+def launch_count() -> int:
+    return int(lib().spiffy_launch_count())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _dev(t: Optional[torch.Tensor], name: str, dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must live on a CUDA device (no CPU path exists)")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise SpiffyError(status, where)
+
+
+def attn_desc(q, k_prefix, k_block, scale=0.0, kernel=ATTN_AUTO) -> AttnDesc:
+    B, N, L, Hq, d = q.shape
+    P = 0 if k_prefix is None else k_prefix.shape[1]
+    Hkv = k_block.shape[3]
+    return AttnDesc(B, N, L, P, Hq, Hkv, d, _dtype_code(q), float(scale), int(kernel))
+
+
+def spiffy_graph_attention_workspace(desc: AttnDesc) -> int:
+    return int(lib().spiffy_graph_attention_workspace(ctypes.byref(desc)))
+
+
+def spiffy_graph_attention(q, k_prefix, v_prefix, k_block, v_block, out=None,
+                           scale: float = 0.0, kernel: int = ATTN_AUTO,
+                           dev_status=None, workspace=None, stream=None):
+    """Packed draft-graph attention.  q [B,N,L,Hq,d]; k/v_prefix [B,P,Hkv,d];
+    k/v_block [B,N,L,Hkv,d]; returns out [B,N,L,Hq,d] (allocated when None)."""
+    desc = attn_desc(q, k_prefix, k_block, scale, kernel)
+    if out is None:
+        out = torch.empty_like(q)
+    need = spiffy_graph_attention_workspace(desc)
+    if need and workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    st = lib().spiffy_graph_attention(
+        ctypes.byref(desc), _dev(q, "q"), _dev(k_prefix, "k_prefix", q.dtype),
+        _dev(v_prefix, "v_prefix", q.dtype), _dev(k_block, "k_block", q.dtype),
+        _dev(v_block, "v_block", q.dtype), _dev(out, "out", q.dtype),
+        _dev(dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
+        ws_bytes, _stream(stream))
+    _check(st, "spiffy_graph_attention")
+    return out
+
+
+def decide_desc(logits, block_tokens, mask_token_id, rule, top_s=1, threshold=0.9) -> DecideDesc:
+    B, N, L = block_tokens.shape
+    V = logits.shape[-1]
+    row_stride = logits.stride(-2) if logits.dim() >= 2 else V
+    return DecideDesc(B, N, L, V, _dtype_code(logits), int(row_stride), int(mask_token_id),
+                      int(rule), int(top_s), float(threshold))
+
+
+def spiffy_unmask_decide_workspace(desc: DecideDesc) -> int:
+    return int(lib().spiffy_unmask_decide_workspace(ctypes.byref(desc)))
+
+
+@dataclass
+class Decision:
+    conf: torch.Tensor         # [B,N,L] float32
+    top_tok: torch.Tensor      # [B,N,L] int32
+    unmask_bits: torch.Tensor  # [B,N] int64 holding the uint64 bit sets
+    n_unmask: torch.Tensor     # [B,N] int32
+    dev_status: torch.Tensor   # [B] int32
+
+
+def _logits_ptr(logits: torch.Tensor) -> int:
+    if not logits.is_cuda:
+        raise ValueError("logits must live on a CUDA device (no CPU path exists)")
+    if logits.stride(-1) != 1:
+        raise ValueError("logits rows must be dense")
+    if logits.dim() == 4:
+        B, N, L, _ = logits.shape
+        rs = logits.stride(2)
+        if (N > 1 and logits.stride(1) != L * rs) or (B > 1 and logits.stride(0) != N * L * rs):
+            raise ValueError("logits rows must be equally spaced")
+    return logits.data_ptr()
+
+
+def spiffy_unmask_decide(logits, block_tokens, mask_token_id: int, rule: int,
+                         top_s: int = 1, threshold: float = 0.9, out: Optional[Decision] = None,
+                         workspace=None, stream=None) -> Decision:
+    """Steps 1-4 of Algorithm 1 for every node.  logits [B,N,L,V] (rows may be
+    a strided view of a wider buffer), block_tokens [B,N,L] int32."""
+    desc = decide_desc(logits, block_tokens, mask_token_id, rule, top_s, threshold)
+    B, N, L = block_tokens.shape
+    dev = logits.device
+    if out is None:
+        out = Decision(torch.empty((B, N, L), dtype=torch.float32, device=dev),
+                       torch.empty((B, N, L), dtype=torch.int32, device=dev),
+                       torch.empty((B, N), dtype=torch.int64, device=dev),
+                       torch.empty((B, N), dtype=torch.int32, device=dev),
+                       torch.zeros((B,), dtype=torch.int32, device=dev))
+    need = spiffy_unmask_decide_workspace(desc)
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    st = lib().spiffy_unmask_decide(
+        ctypes.byref(desc), _logits_ptr(logits), _dev(block_tokens, "block_tokens", torch.int32),
+        _dev(out.conf, "conf", torch.float32), _dev(out.top_tok, "top_tok", torch.int32),
+        _dev(out.unmask_bits, "unmask_bits", torch.int64),
+        _dev(out.n_unmask, "n_unmask", torch.int32),
+        _dev(out.dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
+        workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(st, "spiffy_unmask_decide")
+    return out
+
+
+@dataclass
+class Walk:
+    accepted_node: torch.Tensor  # [B] int32
+    n_accepted: torch.Tensor     # [B] int32
+    path: torch.Tensor           # [B,N] int32
+    next_block: torch.Tensor     # [B,L] int32
+    dev_status: torch.Tensor     # [B] int32
+
+
+def spiffy_accept_walk(block_tokens, parent_off, parent_idx, top_tok, unmask_bits,
+                       out: Optional[Walk] = None, stream=None) -> Walk:
+    """Step 5 of Algorithm 1.  parent_off [B,N+1], parent_idx [B,cap] int32."""
+    B, N, L = block_tokens.shape
+    dev = block_tokens.device
+    desc = DecideDesc(B, N, L, 0, F32, 0, 0, 0, 1, 0.0)
+    if out is None:
+        out = Walk(torch.empty((B,), dtype=torch.int32, device=dev),
+                   torch.empty((B,), dtype=torch.int32, device=dev),
+                   torch.empty((B, N), dtype=torch.int32, device=dev),
+                   torch.empty((B, L), dtype=torch.int32, device=dev),
+                   torch.zeros((B,), dtype=torch.int32, device=dev))
+    if tuple(parent_off.shape) != (B, N + 1) or parent_idx.dim() != 2 or parent_idx.shape[0] != B:
+        raise ValueError("parent_off must be [B,N+1] and parent_idx [B,cap]")
+    st = lib().spiffy_accept_walk(
+        ctypes.byref(desc), _dev(block_tokens, "block_tokens", torch.int32),
+        _dev(parent_off, "parent_off", torch.int32), _dev(parent_idx, "parent_idx", torch.int32),
+        int(parent_idx.shape[1]), _dev(top_tok, "top_tok", torch.int32),
+        _dev(unmask_bits, "unmask_bits", torch.int64),
+        _dev(out.accepted_node, "accepted_node", torch.int32),
+        _dev(out.n_accepted, "n_accepted", torch.int32), _dev(out.path, "path", torch.int32),
+        _dev(out.next_block, "next_block", torch.int32),
+        _dev(out.dev_status, "dev_status", torch.int32), _stream(stream))
+    _check(st, "spiffy_accept_walk")
+    return out

@@ -1,0 +1,105 @@
+"""The C-ABI library without a GPU: it loads, exports every symbol the header
+declares, and turns bad arguments into status codes before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2509_18085_b200 import build as builder
+from paper_2509_18085_b200 import spiffy
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    builder.build()
+    return spiffy.lib()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "spiffy.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(spiffy_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert set(spiffy.EXPORTS) <= set(names)
+    assert len(names) >= 7
+    for name in names:
+        assert getattr(lib, name) is not None
+
+
+def test_status_strings(lib):
+    seen = {lib.spiffy_status_string(i) for i in range(6)}
+    assert len(seen) == 6 and all(seen)
+    assert lib.spiffy_status_string(99)
+
+
+def test_attention_rejects_bad_arguments(lib):
+    fake = ctypes.c_void_p(0x1000)
+    good = spiffy.AttnDesc(1, 2, 8, 16, 4, 2, 64, spiffy.F32, 0.0, spiffy.ATTN_SIMT)
+    call = lambda d, *ptrs: lib.spiffy_graph_attention(ctypes.byref(d), *ptrs, None, None, 0, None)
+    assert call(good, None, fake, fake, fake, fake, fake) == spiffy.EINVAL
+    assert call(good, fake, None, fake, fake, fake, fake) == spiffy.EINVAL  # P > 0 needs a prefix
+    assert call(good, ctypes.c_void_p(0x1004), fake, fake, fake, fake, fake) == spiffy.EINVAL
+    for field, value, want in [("n_kv_heads", 3, spiffy.EINVAL), ("head_dim", 96, spiffy.EUNSUPPORTED),
+                               ("block_len", 65, spiffy.EUNSUPPORTED), ("dtype", 7, spiffy.EINVAL),
+                               ("batch", 0, spiffy.EINVAL), ("prefix_len", -1, spiffy.EINVAL),
+                               ("scale", float("nan"), spiffy.EINVAL), ("kernel", 9, spiffy.EINVAL)]:
+        d = spiffy.AttnDesc(1, 2, 8, 16, 4, 2, 64, spiffy.F32, 0.0, spiffy.ATTN_SIMT)
+        setattr(d, field, value)
+        assert call(d, fake, fake, fake, fake, fake, fake) == want, field
+    # fp32 has no tensor-core kernel
+    d = spiffy.AttnDesc(1, 2, 8, 16, 4, 2, 64, spiffy.F32, 0.0, spiffy.ATTN_TCGEN05)
+    assert call(d, fake, fake, fake, fake, fake, fake) == spiffy.EUNSUPPORTED
+    assert lib.spiffy_graph_attention(None, fake, fake, fake, fake, fake, fake, None, None, 0, None) == spiffy.EINVAL
+
+
+def test_decide_rejects_bad_arguments(lib):
+    fake = ctypes.c_void_p(0x1000)
+
+    def desc(**kw):
+        d = spiffy.DecideDesc(1, 4, 8, 1024, spiffy.BF16, 1024, 1023, spiffy.RULE_TOPS, 1, 0.9)
+        for k, v in kw.items():
+            setattr(d, k, v)
+        return d
+
+    def call(d, ws=fake, ws_bytes=1 << 30, logits=fake):
+        return lib.spiffy_unmask_decide(ctypes.byref(d), logits, fake, fake, fake, fake, fake, None,
+                                        ws, ws_bytes, None)
+
+    assert lib.spiffy_unmask_decide_workspace(ctypes.byref(desc())) > 0
+    assert call(desc(), ws=None) == spiffy.EWORKSPACE
+    assert call(desc(), ws_bytes=8) == spiffy.EWORKSPACE
+    assert call(desc(), logits=None) == spiffy.EINVAL
+    assert call(desc(row_stride=1000)) == spiffy.EINVAL     # shorter than a row
+    assert call(desc(row_stride=1028)) == spiffy.EINVAL     # rows not 16-byte spaced
+    assert call(desc(top_s=0)) == spiffy.EINVAL
+    assert call(desc(rule=5)) == spiffy.EINVAL
+    assert call(desc(block_len=65)) == spiffy.EUNSUPPORTED
+    assert call(desc(vocab=0)) == spiffy.EINVAL
+    assert call(desc(rule=spiffy.RULE_THRESHOLD, threshold=float("nan"))) == spiffy.EINVAL
+    assert lib.spiffy_unmask_decide_workspace(ctypes.byref(desc(vocab=0))) == 0
+
+
+def test_walk_rejects_bad_arguments(lib):
+    fake = ctypes.c_void_p(0x1000)
+    d = spiffy.DecideDesc(1, 4, 8, 0, 0, 0, 0, 0, 1, 0.0)
+    args = [fake] * 3 + [4] + [fake] * 7 + [None]
+    bad = list(args)
+    bad[1] = None
+    assert lib.spiffy_accept_walk(ctypes.byref(d), *bad) == spiffy.EINVAL
+    neg = list(args)
+    neg[3] = -1
+    assert lib.spiffy_accept_walk(ctypes.byref(d), *neg) == spiffy.EINVAL
+
+
+def test_binding_refuses_cpu_tensors():
+    import torch
+    t = torch.zeros(1, 1, 4, 8)
+    tok = torch.zeros(1, 1, 4, dtype=torch.int32)
+    with pytest.raises(ValueError):
+        spiffy.spiffy_unmask_decide(t, tok, 7, spiffy.RULE_TOPS)

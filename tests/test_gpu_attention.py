@@ -1,0 +1,98 @@
+"""GPU parity of spiffy_graph_attention (Sec. 4.3, mask of Fig. 3) with the CPU
+oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2509_18085_b200 import spiffy
+from paper_2509_18085_b200 import workloads as W
+
+import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+KERNELS = [spiffy.ATTN_SIMT, spiffy.ATTN_AUTO]
+
+
+def oracle_attention(w, scale=None):
+    return oracle.graph_attention(w.q, w.k_prefix, w.v_prefix, w.k_block, w.v_block, scale=scale)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("index,n_nodes", [(1, None), (2, None), (3, None), (5, 1), (5, 8), (5, 64)])
+def test_configs(index, n_nodes, kernel):
+    cfg = W.config(index, n_nodes)
+    w = W.make(cfg, W.seed_for(index, 0), decision=False)
+    got = G.gpu_attention(w, kernel)
+    want = oracle_attention(w)
+    assert np.max(np.abs(got - want)) <= G.TOL[cfg.dtype]
+    if cfg.dtype == "bf16":
+        # the result is rounded once to bf16: the error is that rounding
+        assert np.sqrt(np.mean((got - want) ** 2)) < 2e-3
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", [
+    dict(batch=2, n_nodes=3, block_len=5, prefix_len=127, n_q_heads=6, n_kv_heads=2, head_dim=64),
+    dict(batch=1, n_nodes=2, block_len=64, prefix_len=33, n_q_heads=2, n_kv_heads=1, head_dim=128),
+    dict(batch=3, n_nodes=1, block_len=1, prefix_len=0, n_q_heads=1, n_kv_heads=1, head_dim=64),
+    dict(batch=1, n_nodes=5, block_len=16, prefix_len=0, n_q_heads=4, n_kv_heads=4, head_dim=128),
+    dict(batch=2, n_nodes=7, block_len=32, prefix_len=300, n_q_heads=8, n_kv_heads=2, head_dim=128),
+    dict(batch=1, n_nodes=9, block_len=8, prefix_len=1000, n_q_heads=3, n_kv_heads=3, head_dim=128),
+])
+def test_odd_shapes(shape, dtype, kernel):
+    cfg = W.Config("odd", dtype=dtype, vocab=16, rule=0, **shape)
+    w = W.make(cfg, 77, decision=False)
+    got = G.gpu_attention(w, kernel)
+    want = oracle_attention(w)
+    assert np.max(np.abs(got - want)) <= G.TOL[dtype]
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_custom_scale(kernel):
+    cfg = W.config(2, n_nodes=2, prefix_len=200)
+    w = W.make(cfg, 5, decision=False)
+    got = G.gpu_attention(w, kernel, scale=0.05)
+    assert np.max(np.abs(got - oracle_attention(w, scale=0.05))) <= G.TOL["bf16"]
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_packing_invariance_on_the_gpu(kernel):
+    """A draft block's rows must not depend on which other blocks are packed
+    with it (App. A.2): compare the packed call with one call per node."""
+    cfg = W.config(2, n_nodes=5, prefix_len=256)
+    w = W.make(cfg, 9, decision=False)
+    dt = torch.bfloat16
+    q, kp, vp, kb, vb = (G.to_dev(a, dt) for a in (w.q, w.k_prefix, w.v_prefix, w.k_block, w.v_block))
+    packed = spiffy.spiffy_graph_attention(q, kp, vp, kb, vb, kernel=kernel)
+    for n in range(5):
+        alone = spiffy.spiffy_graph_attention(q[:, n:n + 1].contiguous(), kp, vp,
+                                              kb[:, n:n + 1].contiguous(),
+                                              vb[:, n:n + 1].contiguous(), kernel=kernel)
+        diff = (alone[:, 0].float() - packed[:, n].float()).abs().max().item()
+        assert diff <= 2e-2
+    # another node's block must not leak: change node 3's keys, others unchanged bit for bit
+    kb2 = kb.clone()
+    kb2[:, 3] += 1.0
+    again = spiffy.spiffy_graph_attention(q, kp, vp, kb2, vb, kernel=kernel)
+    keep = [0, 1, 2, 4]
+    assert torch.equal(again[:, keep], packed[:, keep])
+    assert not torch.equal(again[:, 3], packed[:, 3])
+
+
+def test_full_size_long_batched_sampled_nodes():
+    """Configuration 4 at full size (B=4, P=4096, N=32): the oracle checks a
+    sample of (sequence, node) pairs one by one, using the fact that a node's
+    output depends only on the context and its own block."""
+    cfg = W.config(4)
+    w = W.make(cfg, W.seed_for(4, 0), decision=False)
+    got = G.gpu_attention(w)
+    rng = np.random.default_rng(0)
+    for _ in range(6):
+        b, n = int(rng.integers(0, cfg.batch)), int(rng.integers(0, cfg.n_nodes))
+        want = oracle.graph_attention(w.q[b:b + 1, n:n + 1], w.k_prefix[b:b + 1], w.v_prefix[b:b + 1],
+                                      w.k_block[b:b + 1, n:n + 1], w.v_block[b:b + 1, n:n + 1])
+        assert np.max(np.abs(got[b, n] - want[0, 0])) <= G.TOL["bf16"]
+    assert np.all(np.isfinite(got))

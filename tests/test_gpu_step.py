@@ -1,0 +1,90 @@
+"""Whole verification steps on the GPU: the full-size decision of the long
+batched configuration on sampled rows, and the losslessness invariant of
+App. A with the CUDA library as the back end of the toy decoder."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import toy
+from paper_2509_18085_b200 import spiffy
+from paper_2509_18085_b200 import workloads as W
+
+import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+def test_full_size_long_batched_decision_sampled():
+    """Configuration 4 at full size: 4 x 32 x 32 rows of 126464 logits.  The
+    oracle evaluates a sample of nodes; the walk is then checked by running
+    the oracle's walk on the GPU's own per-node decisions (integer work)."""
+    cfg = W.config(4)
+    w = W.make(cfg, W.seed_for(4, 0), attention=False)
+    dec, walk = G.gpu_decide(w)
+    conf = dec.conf.cpu().numpy()
+    top = dec.top_tok.cpu().numpy()
+    bits = G.bits_np(dec.unmask_bits)
+    rng = np.random.default_rng(1)
+    for _ in range(12):
+        b, n = int(rng.integers(0, cfg.batch)), int(rng.integers(0, cfg.n_nodes))
+        o = oracle.unmask_decide(w.logits[b:b + 1, n:n + 1], w.block_tokens[b:b + 1, n:n + 1],
+                                 cfg.mask_id, cfg.rule, cfg.top_s, cfg.threshold)
+        masked = w.block_tokens[b, n] == cfg.mask_id
+        assert np.array_equal(top[b, n], o.top_tok[0, 0])
+        assert np.max(np.abs(conf[b, n][masked] - o.conf[0, 0][masked]), initial=0) <= G.TOL["bf16"]
+        if o.margin[0, 0] >= G.MARGIN["bf16"]:
+            assert bits[b, n] == o.unmask_bits[0, 0]
+    # planted winners: with a 4-sigma clip the planted token is the argmax by construction
+    masked = w.block_tokens == cfg.mask_id
+    assert np.array_equal(top[masked], w.planted_tok[masked])
+    sel = (bits[..., None] >> np.arange(cfg.block_len, dtype=np.uint64)) & np.uint64(1)
+    nxt = np.where(sel.astype(bool), top, w.block_tokens).astype(np.int32)
+    ow = oracle.accept_walk(w.block_tokens, w.parent_off, w.parent_idx, nxt, bits)
+    for name in ("accepted_node", "n_accepted", "path", "next_block"):
+        assert np.array_equal(getattr(walk, name).cpu().numpy(), getattr(ow, name)), name
+    assert ow.n_accepted.max() >= 1
+
+
+def gpu_backends(dtype=torch.float32, kernel=spiffy.ATTN_AUTO):
+    def attention(q, kp, vp, kb, vb):
+        t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda().to(dtype)
+        out = spiffy.spiffy_graph_attention(t(q), t(kp), t(vp), t(kb), t(vb), kernel=kernel)
+        return out.float().cpu().numpy()
+
+    def decide(logits, states, mask_id, rule, top_s, threshold):
+        d = spiffy.spiffy_unmask_decide(G.to_dev(logits), G.to_dev(states.astype(np.int32)), mask_id,
+                                        rule, top_s, threshold)
+        return d.top_tok.cpu().numpy(), G.bits_np(d.unmask_bits)
+
+    def walk(states, off, idx, top_tok, unmask_bits, mask_id):
+        g = spiffy.spiffy_accept_walk(G.to_dev(states.astype(np.int32)), G.to_dev(off), G.to_dev(idx),
+                                      G.to_dev(top_tok.astype(np.int32)),
+                                      G.to_dev(unmask_bits.view(np.int64)))
+        return (g.accepted_node.cpu().numpy(), g.n_accepted.cpu().numpy(), g.path.cpu().numpy(),
+                g.next_block.cpu().numpy())
+
+    return attention, decide, walk
+
+
+@pytest.mark.parametrize("rule,S,tau", [(oracle.RULE_TOPS, 1, 0.0), (oracle.RULE_THRESHOLD, 1, 0.8)])
+@pytest.mark.parametrize("seed", range(3))
+def test_losslessness_with_the_cuda_library(rule, S, tau, seed):
+    """Speculative decoding through the CUDA kernels visits exactly the states
+    of plain decoding through the same kernels and saves one model call per
+    accepted draft; both equal the oracle's trajectory."""
+    attention, decide, walk = gpu_backends()
+    start = np.full(8, 23, dtype=np.int32)
+    start[seed] = seed + 1
+    ref_model = toy.ToyModel(seed=seed)
+    ref_traj = toy.vanilla_decode(ref_model, start, rule, S, tau)
+    model = toy.ToyModel(seed=seed, attention=attention)
+    vanilla = toy.vanilla_decode(model, start, rule, S, tau, decide=decide)
+    calls = model.calls
+    assert len(vanilla) == len(ref_traj) and all(np.array_equal(a, b) for a, b in zip(vanilla, ref_traj))
+    drafter = toy.peeking_drafter(vanilla, depth=3, wrong_prob=0.3, seed=seed, vocab=model.vocab)
+    model.calls = 0
+    traj, accepted = toy.speculative_decode(model, start, drafter, rule, S, tau, decide=decide, walk=walk)
+    assert len(traj) == len(vanilla) and all(np.array_equal(a, b) for a, b in zip(traj, vanilla))
+    assert model.calls == calls - sum(accepted)
+    assert sum(accepted) > 0
