@@ -14,7 +14,7 @@ import gpu_util as G
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("index,n_nodes,cases", [(1, None, 10), (2, None, 2), (3, None, 1),
+@pytest.mark.parametrize("index,n_nodes,cases", [(1, None, 10), (2, None, 2), (3, None, 2),
                                                  (5, 1, 2), (5, 8, 1), (5, 64, 1)])
 def test_configs_sharp(index, n_nodes, cases):
     hops = []

@@ -82,9 +82,12 @@ def test_losslessness_with_the_cuda_library(rule, S, tau, seed):
     vanilla = toy.vanilla_decode(model, start, rule, S, tau, decide=decide)
     calls = model.calls
     assert len(vanilla) == len(ref_traj) and all(np.array_equal(a, b) for a, b in zip(vanilla, ref_traj))
-    drafter = toy.peeking_drafter(vanilla, depth=3, wrong_prob=0.3, seed=seed, vocab=model.vocab)
-    model.calls = 0
-    traj, accepted = toy.speculative_decode(model, start, drafter, rule, S, tau, decide=decide, walk=walk)
-    assert len(traj) == len(vanilla) and all(np.array_equal(a, b) for a, b in zip(traj, vanilla))
-    assert model.calls == calls - sum(accepted)
-    assert sum(accepted) > 0
+    total = 0
+    for wrong_prob in (0.3, 0.0):  # spoiled drafts and perfect ones
+        drafter = toy.peeking_drafter(vanilla, depth=3, wrong_prob=wrong_prob, seed=seed, vocab=model.vocab)
+        model.calls = 0
+        traj, accepted = toy.speculative_decode(model, start, drafter, rule, S, tau, decide=decide, walk=walk)
+        assert len(traj) == len(vanilla) and all(np.array_equal(a, b) for a, b in zip(traj, vanilla))
+        assert model.calls == calls - sum(accepted)
+        total += sum(accepted)
+    assert total > 0
