@@ -1,15 +1,540 @@
-// tcgen05/TMEM attention kernel (placeholder until the tensor-core path lands:
-// reports every shape as unsupported, so the CUDA-core kernel is used).
+// Packed draft-graph attention (Sec. 4.3; mask of Fig. 3) on the sm_100a tensor
+// cores: bf16 operands, head dimension 128.
+//
+// Work decomposition.  For one sequence b and one key/value head g, the query
+// rows are all (node n, position l, query head of the group) triples; they all
+// read the same P context keys, and a row of node n additionally reads the L
+// keys of node n's own block.  A CTA owns one M-tile: TNL consecutive (n, l)
+// positions times the `group` query heads of g (TNL = 128 / group, so at most
+// 128 rows), and walks over key tiles of 128 keys: first the context tiles,
+// then the tiles covering the block keys of the nodes its rows belong to.  The
+// mask is never materialised: a context tile is visible to every row, and in a
+// block-key tile row r sees exactly the columns of its own node, a contiguous
+// column range computed from indices.
+//
+// Pipeline inside a CTA (192 threads):
+//   warp 0      TMA producer: Q once, then K and V tiles into two 3-stage rings
+//   warp 1      allocates tensor memory; one lane issues tcgen05.mma:
+//               S = Q K^T (fp32 in TMEM, double buffered), O += P V
+//   warps 2-5   softmax: one thread per row reads S from TMEM, keeps a running
+//               maximum and sum, writes P (bf16) back to TMEM as the A operand
+//               of the second product, rescales O only when the maximum grew by
+//               more than 2^8 (exact: O and the sum always share one reference
+//               maximum), and finally normalises and stores the row.
+// With several splits (grid.z) each CTA handles a slice of the key tiles and
+// stores an unnormalised partial (O, reference maximum, sum); a second kernel
+// merges the partials.
+//
+// Every wait is bounded; a wait that gives up raises SPIFFY_DEV_TIMEOUT in the
+// caller's status word and the CTA winds down without touching its output.
+#include <math.h>
+
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace spiffy {
+namespace {
 
-bool attention_tc_supported(const spiffy_attn_desc&) { return false; }
-size_t attention_tc_workspace_bytes(const spiffy_attn_desc&) { return 0; }
-spiffy_status launch_attention_tc(const spiffy_attn_desc&, const void*, const void*,
-                                  const void*, const void*, const void*, void*,
-                                  int32_t*, void*, cudaStream_t) {
-  return SPIFFY_EUNSUPPORTED;
+using namespace sm100;
+
+constexpr int BM = 128;       // rows of an M-tile (TMEM lanes)
+constexpr int BN = 128;       // keys per key tile
+constexpr int HD = 128;       // head dimension
+constexpr int KS = 3;         // K ring stages
+constexpr int VS = 3;         // V ring stages
+constexpr int kThreads = 192;
+constexpr int kHalfBytes = BN * 128;           // one 64-column half of a tile: 128 rows x 128 B
+constexpr int kTileBytes = 2 * kHalfBytes;     // 32 KB
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColO = 256, kColP = 384;  // S: 2 x 128, O: 128, P: 2 x 64
+constexpr float kRescaleLog2 = 8.0f;
+
+struct Smem {
+  static constexpr int q = 0;
+  static constexpr int k = q + kTileBytes;
+  static constexpr int v = k + KS * kTileBytes;
+  static constexpr int bars = v + VS * kTileBytes;
+  static constexpr int n_bars = 1 + 2 * KS + 2 * VS + 2 + 2 + 1;
+  static constexpr int tmem = bars + 8 * n_bars;
+  static constexpr int abort_flag = tmem + 8;
+  static constexpr int total = abort_flag + 8;
+};
+constexpr int kSmemBytes = Smem::total + 1024;  // slack for 1024-byte alignment
+
+struct Params {
+  int B, N, L, P, Hq, Hkv, group;
+  int TNL;      // (node, position) pairs per M-tile
+  int NL;       // N * L
+  int MT;       // M-tiles per (sequence, kv head)
+  int TP;       // context key tiles
+  int splits;
+  float scale_log2;
+  __nv_bfloat16* out;
+  float* part_o;   // [splits][B*Hkv][MT][128][128]
+  float* part_ml;  // [splits][B*Hkv][MT][128][2]
+  int32_t* status;
+};
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+// Bounded wait that ignores the abort flag (used while winding down).
+__device__ __forceinline__ void mbar_wait_quiet(uint64_t* bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
+                          const __grid_constant__ CUtensorMap tm_kp,
+                          const __grid_constant__ CUtensorMap tm_vp,
+                          const __grid_constant__ CUtensorMap tm_kb,
+                          const __grid_constant__ CUtensorMap tm_vb, const Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  uint8_t* sq = smem + Smem::q;
+  uint8_t* sk = smem + Smem::k;
+  uint8_t* sv = smem + Smem::v;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Smem::bars);
+  uint64_t* q_full = bars;
+  uint64_t* k_full = bars + 1;
+  uint64_t* k_empty = k_full + KS;
+  uint64_t* v_full = k_empty + KS;
+  uint64_t* v_empty = v_full + VS;
+  uint64_t* s_full = v_empty + VS;   // [2]
+  uint64_t* p_ready = s_full + 2;    // [2]
+  uint64_t* pv_done = p_ready + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + Smem::tmem);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + Smem::abort_flag);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int mt = blockIdx.x;
+  const int bg = blockIdx.y;
+  const int b = bg / p.Hkv, g = bg % p.Hkv;
+  const int split = blockIdx.z;
+
+  // this CTA's rows and key tiles
+  const int nl0 = mt * p.TNL;
+  const int nl_count = min(p.TNL, p.NL - nl0);
+  const int rows_box = p.TNL * p.group;        // rows the Q box writes
+  const int rows_valid = nl_count * p.group;   // rows that exist
+  const int n_lo = nl0 / p.L, n_hi = (nl0 + nl_count - 1) / p.L;
+  const int kb_start = n_lo * p.L;
+  const int TB = ((n_hi - n_lo + 1) * p.L + BN - 1) / BN;
+  const int T_all = p.TP + TB;
+  const int t_begin = (int)((int64_t)split * T_all / p.splits);
+  const int t_end = (int)((int64_t)(split + 1) * T_all / p.splits);
+  const int T = t_end - t_begin;
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    for (int i = 0; i < KS; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
+    for (int i = 0; i < VS; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_ready + i, 128); }
+    mbar_init(pv_done, 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  // rows of the Q tile that the TMA box does not write must be finite
+  for (int i = rows_box * 8 + threadIdx.x; i < BM * 8; i += kThreads) {
+    const uint4 z = make_uint4(0, 0, 0, 0);
+    reinterpret_cast<uint4*>(sq)[i] = z;
+    reinterpret_cast<uint4*>(sq + kHalfBytes)[i] = z;
+  }
+  fence_proxy_async_smem();
+  if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ producer --
+    if (lane == 0 && T > 0) {
+      prefetch_tensormap(&tm_q);
+      prefetch_tensormap(p.TP > 0 ? &tm_kp : &tm_kb);
+      mbar_arrive_expect_tx(q_full, 2u * rows_box * 128u);
+      tma_load_4d(sq, &tm_q, q_full, 0, g * p.group, nl0, b);
+      tma_load_4d(sq + kHalfBytes, &tm_q, q_full, 64, g * p.group, nl0, b);
+      int issued_k = 0, issued_v = 0;
+      bool ok = true;
+      auto load = [&](bool is_k, int j) {
+        const int stage = j % (is_k ? KS : VS);
+        const uint32_t round = (uint32_t)(j / (is_k ? KS : VS));
+        uint64_t* empty = (is_k ? k_empty : v_empty) + stage;
+        uint64_t* full = (is_k ? k_full : v_full) + stage;
+        if (!mbar_wait(empty, (round & 1u) ^ 1u, abort_flag)) { ok = false; return; }
+        const int t = t_begin + j;
+        const bool ctx = t < p.TP;
+        const CUtensorMap* m = is_k ? (ctx ? &tm_kp : &tm_kb) : (ctx ? &tm_vp : &tm_vb);
+        const int key0 = ctx ? t * BN : kb_start + (t - p.TP) * BN;
+        uint8_t* dst = (is_k ? sk : sv) + stage * kTileBytes;
+        mbar_arrive_expect_tx(full, kTileBytes);
+        tma_load_4d(dst, m, full, 0, g, key0, b);
+        tma_load_4d(dst + kHalfBytes, m, full, 64, g, key0, b);
+        if (is_k) issued_k = j + 1; else issued_v = j + 1;
+      };
+      load(true, 0);
+      for (int j = 0; j < T && ok; ++j) {
+        if (j + 1 < T) load(true, j + 1);
+        if (ok) load(false, j);
+      }
+      if (!ok) {
+        // winding down: let the copies already in flight land before exit
+        mbar_wait_quiet(q_full, 0);
+        for (int j = max(0, issued_k - KS); j < issued_k; ++j)
+          mbar_wait_quiet(k_full + j % KS, (uint32_t)(j / KS) & 1u);
+        for (int j = max(0, issued_v - VS); j < issued_v; ++j)
+          mbar_wait_quiet(v_full + j % VS, (uint32_t)(j / VS) & 1u);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------- MMA issuer --
+    if (lane == 0 && T > 0) {
+      constexpr uint32_t idesc_s = idesc_bf16_f32(BM, BN, false, false);
+      constexpr uint32_t idesc_o = idesc_bf16_f32(BM, HD, false, true);
+      const uint32_t q_addr = smem_u32(sq);
+      bool ok = mbar_wait(q_full, 0, abort_flag);
+      auto issue_s = [&](int j) {
+        const int stage = j % KS;
+        if (!mbar_wait(k_full + stage, (uint32_t)(j / KS) & 1u, abort_flag)) { ok = false; return; }
+        tc_fence_after_sync();
+        const uint32_t k_addr = smem_u32(sk + stage * kTileBytes);
+        const uint32_t d = tmem + kColS + (uint32_t)(j & 1) * BN;
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk) {
+          const uint32_t off = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
+          umma_ss(d, smem_desc_sw128(q_addr + off, 16, 1024),
+                  smem_desc_sw128(k_addr + off, 16, 1024), idesc_s, kk > 0);
+        }
+        umma_commit(k_empty + stage);
+        umma_commit(s_full + (j & 1));
+      };
+      if (ok) issue_s(0);
+      if (ok && T > 1) issue_s(1);
+      for (int j = 0; j < T && ok; ++j) {
+        const int stage = j % VS;
+        if (!mbar_wait(p_ready + (j & 1), (uint32_t)(j >> 1) & 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(v_full + stage, (uint32_t)(j / VS) & 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after_sync();
+        const uint32_t v_addr = smem_u32(sv + stage * kTileBytes);
+        const uint32_t a = tmem + kColP + (uint32_t)(j & 1) * (BN / 2);
+#pragma unroll
+        for (int kk = 0; kk < BN / 16; ++kk)
+          umma_ts(tmem + kColO, a + 8u * kk,
+                  smem_desc_sw128(v_addr + (uint32_t)kk * 2048u, kHalfBytes, 1024), idesc_o,
+                  (j > 0 || kk > 0) ? 1u : 0u);
+        umma_commit(v_empty + stage);
+        umma_commit(pv_done);
+        if (j + 2 < T) issue_s(j + 2);
+      }
+    }
+  } else if (T > 0) {
+    // ------------------------------------------------------------- softmax --
+    const int quad = warp & 3;               // TMEM lane quadrant this warp may touch
+    const int r = quad * 32 + lane;          // row of the M-tile
+    const bool row_ok = r < rows_valid;
+    const int nl = nl0 + r / p.group;
+    const int hh = r % p.group;
+    const int node = min(nl, p.NL - 1) / p.L;
+    const uint32_t lane_base = (uint32_t)(quad * 32);
+    const float k2 = p.scale_log2;
+    float m_run = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    for (int j = 0; j < T; ++j) {
+      const int buf = j & 1;
+      // wait outcomes are made warp-uniform: the TMEM accesses below are warp-collective
+      if (!__all_sync(0xffffffffu, mbar_wait(s_full + buf, (uint32_t)(j >> 1) & 1u, abort_flag))) {
+        ok = false;
+        break;
+      }
+      tc_fence_after_sync();
+      uint32_t s[BN];
+      tmem_ld_x128(tmem_addr(tmem, lane_base, kColS + (uint32_t)buf * BN), s);
+      // visible columns of this row in this tile: [lo, hi)
+      const int t = t_begin + j;
+      int lo, hi;
+      if (t < p.TP) {
+        lo = 0;
+        hi = min(BN, p.P - t * BN);
+      } else {
+        lo = node * p.L - (kb_start + (t - p.TP) * BN);
+        hi = lo + p.L;
+      }
+      float mx = -INFINITY;
+      if (lo <= 0 && hi >= BN) {
+#pragma unroll
+        for (int c = 0; c < BN; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
+      } else {
+#pragma unroll
+        for (int c = 0; c < BN; ++c) {
+          const float x = (c >= lo && c < hi) ? __uint_as_float(s[c]) : -INFINITY;
+          s[c] = __float_as_uint(x);
+          mx = fmaxf(mx, x);
+        }
+      }
+      const float m_new = fmaxf(m_run, mx * k2);
+      const bool need = (m_new - m_run) > kRescaleLog2;  // false when both are -inf
+      if (__any_sync(0xffffffffu, need)) {
+        float corr = 1.f;
+        if (need) {
+          corr = ex2(m_run - m_new);  // 0 for a row that had seen nothing yet
+          l_run *= corr;
+          m_run = m_new;
+        }
+        if (j > 0) {  // O holds the products of tiles 0..j-1: wait for them, then rescale
+          if (!__all_sync(0xffffffffu, mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, abort_flag))) {
+            ok = false;
+            break;
+          }
+          tc_fence_after_sync();
+#pragma unroll
+          for (int c0 = 0; c0 < HD; c0 += 32) {
+            uint32_t o[32];
+            tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + c0), o);
+#pragma unroll
+            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * corr);
+            tmem_st_x32(tmem_addr(tmem, lane_base, kColO + c0), o);
+          }
+          tmem_wait_st();
+        }
+      }
+      const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+      uint32_t pk[BN / 2];
+      float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+      for (int c = 0; c < BN; c += 2) {
+        const float p0 = ex2(fmaf(__uint_as_float(s[c]), k2, -m_use));
+        const float p1 = ex2(fmaf(__uint_as_float(s[c + 1]), k2, -m_use));
+        sum0 += p0;
+        sum1 += p1;
+        pk[c >> 1] = pack_bf16(p0, p1);
+      }
+      l_run += sum0 + sum1;
+      tmem_st_x64(tmem_addr(tmem, lane_base, kColP + (uint32_t)buf * (BN / 2)), pk);
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(p_ready + buf);
+    }
+    // ------------------------------------------------------------ epilogue --
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(pv_done, (uint32_t)(T - 1) & 1u, abort_flag));
+    if (ok) {
+      tc_fence_after_sync();
+      if (p.splits == 1) {
+        const float inv = 1.0f / l_run;
+        __nv_bfloat16* dst =
+            p.out + (((int64_t)b * p.NL + nl) * p.Hq + (int64_t)g * p.group + hh) * HD;
+#pragma unroll
+        for (int c0 = 0; c0 < HD; c0 += 32) {
+          uint32_t o[32];
+          tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + c0), o);
+          if (row_ok) {
+#pragma unroll
+            for (int c = 0; c < 32; c += 8) {
+              uint4 w;
+              w.x = pack_bf16(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
+              w.y = pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+              w.z = pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+              w.w = pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+              *reinterpret_cast<uint4*>(dst + c0 + c) = w;
+            }
+          }
+        }
+      } else {
+        const int64_t tile = ((int64_t)split * gridDim.y + bg) * p.MT + mt;
+        float* po = p.part_o + (tile * BM + r) * HD;
+        float* pml = p.part_ml + (tile * BM + r) * 2;
+#pragma unroll
+        for (int c0 = 0; c0 < HD; c0 += 32) {
+          uint32_t o[32];
+          tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + c0), o);
+          if (row_ok) {
+#pragma unroll
+            for (int c = 0; c < 32; c += 4)
+              *reinterpret_cast<uint4*>(po + c0 + c) = make_uint4(o[c], o[c + 1], o[c + 2], o[c + 3]);
+          }
+        }
+        if (row_ok) {
+          pml[0] = m_run;
+          pml[1] = l_run;
+        }
+      }
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem, kTmemCols);
+  }
+  if (threadIdx.x == 0 && *abort_flag && p.status) atomicOr(p.status, SPIFFY_DEV_TIMEOUT);
+}
+
+// Merge of the per-split partials: one warp per output row, lane = 4 columns.
+__global__ void __launch_bounds__(256)
+graph_attention_combine_kernel(const Params p) {
+  const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);  // (b, nl, h)
+  const int lane = threadIdx.x & 31;
+  const int64_t rows = (int64_t)p.B * p.NL * p.Hq;
+  if (row >= rows) return;
+  const int h = (int)(row % p.Hq);
+  const int nl = (int)((row / p.Hq) % p.NL);
+  const int b = (int)(row / ((int64_t)p.Hq * p.NL));
+  const int g = h / p.group, hh = h % p.group;
+  const int mt = nl / p.TNL;
+  const int r = (nl - mt * p.TNL) * p.group + hh;
+  const int64_t BG = (int64_t)p.B * p.Hkv;
+  float M = -INFINITY;
+  for (int s = 0; s < p.splits; ++s) {
+    const int64_t tile = ((int64_t)s * BG + (int64_t)b * p.Hkv + g) * p.MT + mt;
+    M = fmaxf(M, p.part_ml[(tile * BM + r) * 2]);
+  }
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float l = 0.f;
+  for (int s = 0; s < p.splits; ++s) {
+    const int64_t tile = ((int64_t)s * BG + (int64_t)b * p.Hkv + g) * p.MT + mt;
+    const float m = p.part_ml[(tile * BM + r) * 2];
+    if (m == -INFINITY) continue;  // this slice held no visible key for the row
+    const float w = ex2(m - M);
+    l += w * p.part_ml[(tile * BM + r) * 2 + 1];
+    const float4 o = *reinterpret_cast<const float4*>(p.part_o + (tile * BM + r) * HD + lane * 4);
+    acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
+  }
+  const float inv = 1.0f / l;
+  uint2 w2;
+  w2.x = pack_bf16(acc.x * inv, acc.y * inv);
+  w2.y = pack_bf16(acc.z * inv, acc.w * inv);
+  *reinterpret_cast<uint2*>(p.out + row * HD + lane * 4) = w2;
+}
+
+// ------------------------------------------------------------------ host ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess)
+      f = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(f);
+  }();
+  return fn;
+}
+
+// Tensor [outer][rows][heads][128] of bf16 seen as a 4-D TMA tensor with the
+// 64-element half of a head row innermost; box = 64 x box_heads x box_rows x 1.
+bool make_map(CUtensorMap* m, const void* base, int heads, int64_t rows, int outer, int box_heads,
+              int box_rows) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return false;
+  const cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)heads, (cuuint64_t)rows, (cuuint64_t)outer};
+  const cuuint64_t strides[3] = {(cuuint64_t)HD * 2, (cuuint64_t)heads * HD * 2,
+                                 (cuuint64_t)rows * heads * HD * 2};
+  const cuuint32_t box[4] = {64, (cuuint32_t)box_heads, (cuuint32_t)box_rows, 1};
+  const cuuint32_t es[4] = {1, 1, 1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+             es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct Plan {
+  int group, TNL, NL, MT, TP, splits;
+  int64_t tiles;  // B * Hkv * MT
+};
+
+Plan make_plan(const spiffy_attn_desc& d) {
+  Plan pl;
+  pl.group = d.n_q_heads / d.n_kv_heads;
+  pl.TNL = BM / pl.group;
+  pl.NL = d.n_nodes * d.block_len;
+  pl.MT = (pl.NL + pl.TNL - 1) / pl.TNL;
+  pl.TP = (d.prefix_len + BN - 1) / BN;
+  pl.tiles = (int64_t)d.batch * d.n_kv_heads * pl.MT;
+  // Fewer CTAs than SMs: cut the key tiles of each M-tile into slices so that
+  // the context streams through more SMs at once.
+  int splits = 1;
+  if (pl.tiles < 120) {
+    splits = (int)(148 / pl.tiles);
+    if (splits > pl.TP + 1) splits = pl.TP + 1;
+    if (splits < 1) splits = 1;
+  }
+  pl.splits = splits;
+  return pl;
+}
+
+}  // namespace
+
+bool attention_tc_supported(const spiffy_attn_desc& d) {
+  if (d.dtype != SPIFFY_BF16 || d.head_dim != HD) return false;
+  const int group = d.n_q_heads / d.n_kv_heads;
+  if (group > BM) return false;
+  if ((int64_t)d.batch * d.n_kv_heads > 65535) return false;
+  return true;
+}
+
+size_t attention_tc_workspace_bytes(const spiffy_attn_desc& d) {
+  const Plan pl = make_plan(d);
+  if (pl.splits == 1) return 0;
+  return (size_t)pl.splits * pl.tiles * BM * (HD + 2) * sizeof(float);
+}
+
+spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q, const void* kp,
+                                  const void* vp, const void* kb, const void* vb, void* out,
+                                  int32_t* dev_status, void* ws, cudaStream_t stream) {
+  const Plan pl = make_plan(d);
+  CUtensorMap tm_q, tm_kp, tm_vp, tm_kb, tm_vb;
+  bool ok = make_map(&tm_q, q, d.n_q_heads, pl.NL, d.batch, pl.group, pl.TNL);
+  ok = ok && make_map(&tm_kb, kb, d.n_kv_heads, pl.NL, d.batch, 1, BN);
+  ok = ok && make_map(&tm_vb, vb, d.n_kv_heads, pl.NL, d.batch, 1, BN);
+  if (d.prefix_len > 0) {
+    ok = ok && make_map(&tm_kp, kp, d.n_kv_heads, d.prefix_len, d.batch, 1, BN);
+    ok = ok && make_map(&tm_vp, vp, d.n_kv_heads, d.prefix_len, d.batch, 1, BN);
+  } else {  // never dereferenced: there is no context tile
+    tm_kp = tm_kb;
+    tm_vp = tm_vb;
+  }
+  if (!ok) return SPIFFY_ECUDA;
+
+  Params p;
+  p.B = d.batch; p.N = d.n_nodes; p.L = d.block_len; p.P = d.prefix_len;
+  p.Hq = d.n_q_heads; p.Hkv = d.n_kv_heads; p.group = pl.group;
+  p.TNL = pl.TNL; p.NL = pl.NL; p.MT = pl.MT; p.TP = pl.TP; p.splits = pl.splits;
+  const float scale = d.scale != 0.f ? d.scale : 1.0f / sqrtf((float)d.head_dim);
+  p.scale_log2 = scale * kLog2e;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.part_o = static_cast<float*>(ws);
+  p.part_ml = p.part_o ? p.part_o + (size_t)pl.splits * pl.tiles * BM * HD : nullptr;
+  p.status = dev_status;
+
+  if (cudaFuncSetAttribute(graph_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kSmemBytes) != cudaSuccess)
+    return SPIFFY_ECUDA;
+  const dim3 grid(pl.MT, d.batch * d.n_kv_heads, pl.splits);
+  graph_attention_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_kp, tm_vp, tm_kb,
+                                                                    tm_vb, p);
+  count_launch();
+  if (cudaGetLastError() != cudaSuccess) return SPIFFY_ECUDA;
+  if (pl.splits > 1) {
+    const int64_t rows = (int64_t)d.batch * pl.NL * d.n_q_heads;
+    graph_attention_combine_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, stream>>>(p);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return SPIFFY_ECUDA;
+  }
+  return SPIFFY_OK;
 }
 
 }  // namespace spiffy

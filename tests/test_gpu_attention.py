@@ -12,7 +12,23 @@ import gpu_util as G
 
 pytestmark = pytest.mark.gpu
 
-KERNELS = [spiffy.ATTN_SIMT, spiffy.ATTN_AUTO]
+KERNELS = [spiffy.ATTN_SIMT, spiffy.ATTN_AUTO, spiffy.ATTN_TCGEN05]
+
+
+def tc_takes(cfg):
+    """The tensor-core kernel takes bf16 inputs with head dimension 128."""
+    return cfg.dtype == "bf16" and cfg.head_dim == 128 and cfg.n_q_heads // cfg.n_kv_heads <= 128
+
+
+def run_or_expect_unsupported(w, kernel, **kw):
+    """Forcing the tensor-core kernel on a shape it does not take must be
+    refused with a status code, never silently served by another kernel."""
+    if kernel == spiffy.ATTN_TCGEN05 and not tc_takes(w.cfg):
+        with pytest.raises(spiffy.SpiffyError) as e:
+            G.gpu_attention(w, kernel, **kw)
+        assert e.value.status == spiffy.EUNSUPPORTED
+        return None
+    return G.gpu_attention(w, kernel, **kw)
 
 
 def oracle_attention(w, scale=None):
@@ -24,7 +40,9 @@ def oracle_attention(w, scale=None):
 def test_configs(index, n_nodes, kernel):
     cfg = W.config(index, n_nodes)
     w = W.make(cfg, W.seed_for(index, 0), decision=False)
-    got = G.gpu_attention(w, kernel)
+    got = run_or_expect_unsupported(w, kernel)
+    if got is None:
+        return
     want = oracle_attention(w)
     assert np.max(np.abs(got - want)) <= G.TOL[cfg.dtype]
     if cfg.dtype == "bf16":
@@ -45,7 +63,9 @@ def test_configs(index, n_nodes, kernel):
 def test_odd_shapes(shape, dtype, kernel):
     cfg = W.Config("odd", dtype=dtype, vocab=16, rule=0, **shape)
     w = W.make(cfg, 77, decision=False)
-    got = G.gpu_attention(w, kernel)
+    got = run_or_expect_unsupported(w, kernel)
+    if got is None:
+        return
     want = oracle_attention(w)
     assert np.max(np.abs(got - want)) <= G.TOL[dtype]
 
