@@ -219,25 +219,23 @@ def main():
 
     import numpy as np
     import torch
-    import torch.distributed as dist
-
+    from paper_2509_18085_b200 import replicas
     from paper_2509_18085_b200 import spiffy
     from paper_2509_18085_b200 import workloads as W
     from paper_2509_18085_b200.step import VerifyStep, inputs_from_workload
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    ranks = replicas.from_env()
+    world, rank, local = ranks.world, ranks.rank, ranks.local
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    replicas.init(ranks, "nccl", torch.device("cuda", local))
     spiffy.lib()  # fail loudly now if the library is missing
 
     cfg = W.config(args.config, args.nodes)
     kernel = {"auto": spiffy.ATTN_AUTO, "simt": spiffy.ATTN_SIMT, "tcgen05": spiffy.ATTN_TCGEN05}[args.attn_kernel]
-    work = [W.make(cfg, W.seed_for(args.config, 100 + i + rank * N_SETS)) for i in range(N_SETS)]
+    first_case = 100 + replicas.case_offset(ranks, N_SETS)
+    work = [W.make(cfg, W.seed_for(args.config, first_case + i)) for i in range(N_SETS)]
     sets = [inputs_from_workload(w) for w in work]
     host0 = inputs_from_workload(work[0], device="cpu", pin=True)
     step = VerifyStep(cfg, attn_kernel=kernel)
@@ -266,8 +264,7 @@ def main():
         for _ in range(warm_replays):
             graph.replay()
         stream.synchronize()
-        if world > 1:
-            dist.barrier()
+        replicas.barrier(ranks)
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
@@ -275,8 +272,7 @@ def main():
             graph.replay()
         e1.record(stream)
         stream.synchronize()
-        if world > 1:
-            dist.barrier()
+        replicas.barrier(ranks)
         torch.cuda.synchronize()
         ms_total = e0.elapsed_time(e1)
 
@@ -318,13 +314,10 @@ def main():
             int(step.walk.dev_status.max().item())
 
     # max over ranks
-    t = torch.tensor([ms_total, ms_e2e], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_total, ms_e2e = replicas.max_over_ranks(ranks, [ms_total, ms_e2e], device="cuda")
     ms_per_step = ms_total / steps
-    value = world * steps / (ms_total * 1e-3)
-    e2e_value = world / (ms_e2e * 1e-3)
+    value = replicas.whole_job_rate(ranks, steps, ms_total)
+    e2e_value = replicas.whole_job_rate(ranks, 1, ms_e2e)
 
     peaks = measured_peaks()
     roofline = {
@@ -370,8 +363,7 @@ def main():
                                 "sample": f"median of 5 full steps of the same workload ({what})"}
     if rank == 0:
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.finish(ranks)
 
 
 if __name__ == "__main__":
