@@ -170,6 +170,47 @@ spiffy_status spiffy_unmask_decide(const spiffy_decide_desc* desc,
                                    void* workspace, size_t workspace_bytes,
                                    void* cuda_stream);
 
+/*
+ * The same decision step for callers that cannot provide scratch memory.  (The
+ * paper has no counterpart: this is a packaging variant of the call above.)
+ *
+ * Who needs it: code that must not, or cannot, allocate device memory when it
+ * calls -- a plug-in inside a serving engine that has already claimed the
+ * whole device for its own pool, so that cudaMalloc would fail; a decode loop
+ * whose latency budget does not tolerate cudaMalloc's device-wide
+ * synchronisation; a caller that simply has no allocator at hand.  Such a
+ * caller still passes its inputs and outputs, but no workspace: the partial
+ * results of the vocabulary reduction go to one fixed array of
+ * SPIFFY_DECIDE_STATIC_BYTES bytes that is part of the library image (every GPU
+ * on which the library is loaded holds that array until the process exits).
+ * The call performs no cudaMalloc, cudaFree or other allocation.
+ *
+ * Arguments, layouts, results and status bits are those of
+ * spiffy_unmask_decide.  Differences:
+ *   - A shape whose scratch need (spiffy_unmask_decide_workspace) exceeds
+ *     SPIFFY_DECIDE_STATIC_BYTES is refused with SPIFFY_EUNSUPPORTED and nothing
+ *     is launched.  The limit (512 KiB) covers every benchmark shape, the
+ *     largest being B*N*L = 4096 rows; batches of several ten thousand rows
+ *     go beyond it and have to use the regular entry point.
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current) and keeps it; make that
+ *     first call outside any stream capture.
+ *   - All calls in the process share the one array, and it keeps whatever the
+ *     last call left.  Nothing in it needs clearing between calls, but two
+ *     calls that overlap on the GPU (different streams, or one device used
+ *     from two threads without ordering) race on it and give undefined
+ *     results: order them on one stream or with events.
+ */
+#define SPIFFY_DECIDE_STATIC_BYTES (512u << 10)
+spiffy_status spiffy_unmask_decide_static(const spiffy_decide_desc* desc,
+                                          const void* logits,
+                                          const int32_t* block_tokens,
+                                          float* conf, int32_t* top_tok,
+                                          uint64_t* unmask_bits,
+                                          int32_t* n_unmask,
+                                          int32_t* dev_status,
+                                          void* cuda_stream);
+
 /* ------------------------------------------------------------------------- */
 /* Acceptance: step 5 of Algorithm 1 over the draft graph of Sec. 4.4.1      */
 /* ------------------------------------------------------------------------- */

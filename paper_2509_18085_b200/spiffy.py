@@ -27,7 +27,9 @@ EXPORTS = (
     "spiffy_graph_attention_workspace", "spiffy_graph_attention",
     "spiffy_unmask_decide_workspace", "spiffy_unmask_decide",
     "spiffy_accept_walk", "spiffy_status_string", "spiffy_launch_count",
+    "spiffy_unmask_decide_static",
 )
+DECIDE_STATIC_BYTES = 512 << 10
 
 
 class SpiffyError(RuntimeError):
@@ -74,6 +76,8 @@ def lib() -> ctypes.CDLL:
         L.spiffy_unmask_decide_workspace.argtypes = [ctypes.POINTER(DecideDesc)]
         L.spiffy_unmask_decide.restype = ctypes.c_int
         L.spiffy_unmask_decide.argtypes = [ctypes.POINTER(DecideDesc)] + [vp] * 8 + [sz, vp]
+        L.spiffy_unmask_decide_static.restype = ctypes.c_int
+        L.spiffy_unmask_decide_static.argtypes = [ctypes.POINTER(DecideDesc)] + [vp] * 8
         L.spiffy_accept_walk.restype = ctypes.c_int
         L.spiffy_accept_walk.argtypes = [ctypes.POINTER(DecideDesc), vp, vp, vp, i32] + [vp] * 8
         L.spiffy_status_string.restype = ctypes.c_char_p
@@ -210,6 +214,25 @@ def spiffy_unmask_decide(logits, block_tokens, mask_token_id: int, rule: int,
         _dev(out.dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
         workspace.numel() * workspace.element_size(), _stream(stream))
     _check(st, "spiffy_unmask_decide")
+    return out
+
+
+def spiffy_unmask_decide_static(logits, block_tokens, mask_token_id: int, rule: int, out: Decision,
+                                top_s: int = 1, threshold: float = 0.9, stream=None) -> Decision:
+    """The decision step without any workspace: scratch lives in a fixed array
+    inside the library (``DECIDE_STATIC_BYTES``), for callers that cannot
+    allocate device memory at call time.  ``out`` must be preallocated by the
+    caller -- this wrapper allocates nothing either.  Calls that overlap on the
+    GPU share that array and race; shapes that need more scratch raise
+    ``SpiffyError`` with status ``EUNSUPPORTED``."""
+    desc = decide_desc(logits, block_tokens, mask_token_id, rule, top_s, threshold)
+    st = lib().spiffy_unmask_decide_static(
+        ctypes.byref(desc), _logits_ptr(logits), _dev(block_tokens, "block_tokens", torch.int32),
+        _dev(out.conf, "conf", torch.float32), _dev(out.top_tok, "top_tok", torch.int32),
+        _dev(out.unmask_bits, "unmask_bits", torch.int64),
+        _dev(out.n_unmask, "n_unmask", torch.int32),
+        _dev(out.dev_status, "dev_status", torch.int32), _stream(stream))
+    _check(st, "spiffy_unmask_decide_static")
     return out
 
 
