@@ -157,6 +157,8 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
+  // everything above is on-chip set-up; global memory is touched from here on
+  cudaGridDependencySynchronize();
 
   if (warp == 0) {
     // ------------------------------------------------------------ producer --
@@ -384,6 +386,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
 // Merge of the per-split partials: one warp per output row, lane = 4 columns.
 __global__ void __launch_bounds__(256)
 graph_attention_combine_kernel(const Params p) {
+  cudaGridDependencySynchronize();  // the partials are visible
   const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);  // (b, nl, h)
   const int lane = threadIdx.x & 31;
   const int64_t rows = (int64_t)p.B * p.NL * p.Hq;
@@ -524,15 +527,16 @@ spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q, cons
                            kSmemBytes) != cudaSuccess)
     return SPIFFY_ECUDA;
   const dim3 grid(pl.MT, d.batch * d.n_kv_heads, pl.splits);
-  graph_attention_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_kp, tm_vp, tm_kb,
-                                                                    tm_vb, p);
+  if (launch_pdl(graph_attention_tc_kernel, grid, dim3(kThreads), (size_t)kSmemBytes, stream, tm_q,
+                 tm_kp, tm_vp, tm_kb, tm_vb, p) != cudaSuccess)
+    return SPIFFY_ECUDA;
   count_launch();
-  if (cudaGetLastError() != cudaSuccess) return SPIFFY_ECUDA;
   if (pl.splits > 1) {
     const int64_t rows = (int64_t)d.batch * pl.NL * d.n_q_heads;
-    graph_attention_combine_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, stream>>>(p);
+    if (launch_pdl(graph_attention_combine_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256),
+                   (size_t)0, stream, p) != cudaSuccess)
+      return SPIFFY_ECUDA;
     count_launch();
-    if (cudaGetLastError() != cudaSuccess) return SPIFFY_ECUDA;
   }
   return SPIFFY_OK;
 }

@@ -46,6 +46,26 @@ spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q,
                                   int32_t* dev_status, void* ws,
                                   cudaStream_t stream);
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled
+// while its predecessor in the stream is still draining.  Every kernel launched
+// this way calls cudaGridDependencySynchronize() before it touches global
+// memory, so its reads and writes are ordered after the predecessor.
+template <typename... Args>
+cudaError_t launch_pdl(void (*kern)(Args...), dim3 grid, dim3 block, size_t smem,
+                       cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
 inline spiffy_status check_launch() {
   return cudaGetLastError() == cudaSuccess ? SPIFFY_OK : SPIFFY_ECUDA;
 }

@@ -135,6 +135,9 @@ decide_reduce_kernel(const T* __restrict__ logits, int64_t row_stride, int V,
                      int64_t chunk, int splits,
                      const int32_t* __restrict__ block_tokens, int mask_id,
                      Partial* __restrict__ partials) {
+#if __CUDA_ARCH__ >= 900
+  cudaGridDependencySynchronize();  // inputs written by earlier kernels are visible
+#endif
   const int row = blockIdx.y;
   if (block_tokens[row] != mask_id) return;  // already unmasked: never read
   const int split = blockIdx.x;
@@ -287,36 +290,25 @@ spiffy_status launch_decide(const spiffy_decide_desc& d, const void* logits,
   const int rows = d.batch * d.n_nodes * d.block_len;
   Partial* partials = static_cast<Partial*>(ws);
   const dim3 grid(splits, rows);
-  if (d.logits_dtype == SPIFFY_BF16) {
-    decide_reduce_kernel<__nv_bfloat16><<<grid, kReduceThreads, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(logits), d.row_stride, d.vocab, chunk,
-        splits, block_tokens, d.mask_token_id, partials);
-  } else {
-    decide_reduce_kernel<float><<<grid, kReduceThreads, 0, stream>>>(
-        static_cast<const float*>(logits), d.row_stride, d.vocab, chunk, splits,
-        block_tokens, d.mask_token_id, partials);
-  }
+  cudaError_t e;
+  if (d.logits_dtype == SPIFFY_BF16)
+    e = launch_pdl(decide_reduce_kernel<__nv_bfloat16>, grid, dim3(kReduceThreads), (size_t)0, stream,
+                   static_cast<const __nv_bfloat16*>(logits), (int64_t)d.row_stride, (int)d.vocab,
+                   chunk, splits, block_tokens, (int)d.mask_token_id, partials);
+  else
+    e = launch_pdl(decide_reduce_kernel<float>, grid, dim3(kReduceThreads), (size_t)0, stream,
+                   static_cast<const float*>(logits), (int64_t)d.row_stride, (int)d.vocab, chunk,
+                   splits, block_tokens, (int)d.mask_token_id, partials);
   count_launch();
-  if (cudaGetLastError() != cudaSuccess) return SPIFFY_ECUDA;
+  if (e != cudaSuccess) return SPIFFY_ECUDA;
 
-  // The finalize kernel is launched with programmatic stream serialisation:
-  // its launch overlaps the tail of the reduce kernel and it waits on the
-  // device (cudaGridDependencySynchronize) for the partials.
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(d.batch * d.n_nodes);
-  cfg.blockDim = dim3(64);
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  // The finalize kernel's launch overlaps the tail of the reduce kernel; it
+  // waits on the device (cudaGridDependencySynchronize) for the partials.
   const Partial* cpart = partials;
-  cudaError_t e = cudaLaunchKernelEx(
-      &cfg, decide_finalize_kernel, cpart, splits, (int)d.n_nodes,
-      (int)d.block_len, block_tokens, (int)d.mask_token_id, (int)d.rule,
-      (int)d.top_s, d.threshold, conf, top_tok, unmask_bits, n_unmask,
-      dev_status);
+  e = launch_pdl(decide_finalize_kernel, dim3(d.batch * d.n_nodes), dim3(64), (size_t)0, stream,
+                 cpart, splits, (int)d.n_nodes, (int)d.block_len, block_tokens,
+                 (int)d.mask_token_id, (int)d.rule, (int)d.top_s, d.threshold, conf, top_tok,
+                 unmask_bits, n_unmask, dev_status);
   count_launch();
   return e == cudaSuccess ? SPIFFY_OK : SPIFFY_ECUDA;
 }

@@ -14,7 +14,10 @@ accept_walk_kernel(int N, int L, const int32_t* __restrict__ block_tokens,
                    int32_t* __restrict__ accepted_node,
                    int32_t* __restrict__ n_accepted, int32_t* __restrict__ path,
                    int32_t* __restrict__ next_block,
-                   int32_t* __restrict__ dev_status) {
+                   int32_t* __restrict__ dev_status, int stage_in_smem) {
+#if __CUDA_ARCH__ >= 900
+  cudaGridDependencySynchronize();  // the decision kernel's outputs are visible
+#endif
   const int b = blockIdx.x;
   const int lane = threadIdx.x;
   const unsigned full = 0xffffffffu;
@@ -22,6 +25,23 @@ accept_walk_kernel(int N, int L, const int32_t* __restrict__ block_tokens,
   const int32_t* top = top_tok + (int64_t)b * N * L;
   const int32_t* off = parent_off + (int64_t)b * (N + 1);
   const int32_t* idx = parent_idx + (int64_t)b * parent_cap;
+  const uint64_t* ubits = unmask_bits + (int64_t)b * N;
+  // The walk is a chain of dependent reads: when the sequence's graph fits,
+  // copy it to shared memory first (all loads in flight at once) and walk there.
+  extern __shared__ __align__(8) unsigned char walk_smem[];
+  if (stage_in_smem) {
+    uint64_t* s_bits = reinterpret_cast<uint64_t*>(walk_smem);
+    int32_t* s_state = reinterpret_cast<int32_t*>(s_bits + N);
+    int32_t* s_top = s_state + N * L;
+    int32_t* s_off = s_top + N * L;
+    int32_t* s_idx = s_off + (N + 1);
+    for (int i = lane; i < N * L; i += 32) { s_state[i] = state[i]; s_top[i] = top[i]; }
+    for (int i = lane; i <= N; i += 32) s_off[i] = off[i];
+    for (int i = lane; i < parent_cap; i += 32) s_idx[i] = idx[i];
+    for (int i = lane; i < N; i += 32) s_bits[i] = ubits[i];
+    __syncwarp();
+    state = s_state; top = s_top; off = s_off; idx = s_idx; ubits = s_bits;
+  }
   int32_t* pth = path + (int64_t)b * N;
   for (int i = lane; i < N; i += 32) pth[i] = i == 0 ? 0 : -1;
   const int l0 = lane, l1 = lane + 32;
@@ -32,7 +52,7 @@ accept_walk_kernel(int N, int L, const int32_t* __restrict__ block_tokens,
     if (l >= L) return 0;
     return ((bits >> l) & 1ull) ? top[node * L + l] : state[node * L + l];
   };
-  uint64_t bits = unmask_bits[(int64_t)b * N];
+  uint64_t bits = ubits[0];
   int32_t nx0 = next_of(0, bits, l0), nx1 = next_of(0, bits, l1);
   while (hops < N - 1 && bits != 0) {
     int found = -1;
@@ -59,7 +79,7 @@ accept_walk_kernel(int N, int L, const int32_t* __restrict__ block_tokens,
     cur = found;  // accepted: its distribution replaces the target's
     ++hops;
     if (lane == 0) pth[hops] = cur;
-    bits = unmask_bits[(int64_t)b * N + cur];
+    bits = ubits[cur];
     nx0 = next_of(cur, bits, l0);
     nx1 = next_of(cur, bits, l1);
   }
@@ -83,12 +103,16 @@ spiffy_status launch_walk(const spiffy_decide_desc& d,
                           int32_t* n_accepted, int32_t* path,
                           int32_t* next_block, int32_t* dev_status,
                           cudaStream_t stream) {
-  accept_walk_kernel<<<d.batch, 32, 0, stream>>>(
-      d.n_nodes, d.block_len, block_tokens, parent_off, parent_idx, parent_cap,
-      top_tok, unmask_bits, accepted_node, n_accepted, path, next_block,
-      dev_status);
+  const size_t need = (size_t)d.n_nodes * 8 +
+                      ((size_t)2 * d.n_nodes * d.block_len + d.n_nodes + 1 + parent_cap) * 4;
+  const int stage_in_smem = need <= 40 * 1024;
+  const cudaError_t e = launch_pdl(
+      accept_walk_kernel, dim3(d.batch), dim3(32), stage_in_smem ? need : (size_t)0, stream,
+      (int)d.n_nodes, (int)d.block_len, block_tokens, parent_off, parent_idx, (int)parent_cap,
+      top_tok, unmask_bits, accepted_node, n_accepted, path, next_block, dev_status,
+      stage_in_smem);
   count_launch();
-  return check_launch();
+  return e == cudaSuccess ? SPIFFY_OK : SPIFFY_ECUDA;
 }
 
 }  // namespace spiffy
