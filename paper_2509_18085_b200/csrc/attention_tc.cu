@@ -12,15 +12,19 @@
 // block-key tile row r sees exactly the columns of its own node, a contiguous
 // column range computed from indices.
 //
-// Pipeline inside a CTA (192 threads):
+// Pipeline inside a CTA (320 threads):
 //   warp 0      TMA producer: Q once, then K and V tiles into two 3-stage rings
 //   warp 1      allocates tensor memory; one lane issues tcgen05.mma:
 //               S = Q K^T (fp32 in TMEM, double buffered), O += P V
-//   warps 2-5   softmax: one thread per row reads S from TMEM, keeps a running
-//               maximum and sum, writes P (bf16) back to TMEM as the A operand
-//               of the second product, rescales O only when the maximum grew by
-//               more than 2^8 (exact: O and the sum always share one reference
-//               maximum), and finally normalises and stores the row.
+//   warps 2-9   two softmax warpgroups; the first takes the even key tiles, the
+//               second the odd ones, each with its own S buffer, accumulator O
+//               and running (maximum, sum), so that the exponentials of one
+//               tile overlap the other tile's products.  One thread per row
+//               reads S from TMEM, writes P (bf16) back over it as the A
+//               operand of the second product, and rescales its O only when
+//               the maximum grew by more than 2^8 (exact: O and the sum always
+//               share one reference maximum).  At the end the two accumulators
+//               are merged, normalised and stored.
 // With several splits (grid.z) each CTA handles a slice of the key tiles and
 // stores an unnormalised partial (O, reference maximum, sum); a second kernel
 // merges the partials.
@@ -42,11 +46,13 @@ constexpr int BN = 128;       // keys per key tile
 constexpr int HD = 128;       // head dimension
 constexpr int KS = 3;         // K ring stages
 constexpr int VS = 3;         // V ring stages
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;  // producer warp, MMA warp, two softmax warpgroups
 constexpr int kHalfBytes = BN * 128;           // one 64-column half of a tile: 128 rows x 128 B
 constexpr int kTileBytes = 2 * kHalfBytes;     // 32 KB
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColO = 256, kColP = 384;  // S: 2 x 128, O: 128, P: 2 x 64
+// S: 2 x 128 columns (P, as bf16 pairs, overwrites the first 64 columns of its S);
+// O: 2 x 128 columns, one accumulator per softmax warpgroup
+constexpr uint32_t kColS = 0, kColO = 256;
 constexpr float kRescaleLog2 = 8.0f;
 
 struct Smem {
@@ -54,7 +60,7 @@ struct Smem {
   static constexpr int k = q + kTileBytes;
   static constexpr int v = k + KS * kTileBytes;
   static constexpr int bars = v + VS * kTileBytes;
-  static constexpr int n_bars = 1 + 2 * KS + 2 * VS + 2 + 2 + 1;
+  static constexpr int n_bars = 1 + 2 * KS + 2 * VS + 2 + 2 + 2;
   static constexpr int tmem = bars + 8 * n_bars;
   static constexpr int abort_flag = tmem + 8;
   static constexpr int total = abort_flag + 8;
@@ -113,7 +119,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
   uint64_t* v_empty = v_full + VS;
   uint64_t* s_full = v_empty + VS;   // [2]
   uint64_t* p_ready = s_full + 2;    // [2]
-  uint64_t* pv_done = p_ready + 2;
+  uint64_t* pv_done = p_ready + 2;   // [2], one per softmax warpgroup
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + Smem::tmem);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + Smem::abort_flag);
 
@@ -142,6 +148,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     for (int i = 0; i < VS; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_ready + i, 128); }
     mbar_init(pv_done, 1);
+    mbar_init(pv_done + 1, 1);
     *abort_flag = 0;
     mbar_fence_init();
   }
@@ -230,39 +237,43 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         if (!mbar_wait(v_full + stage, (uint32_t)(j / VS) & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t v_addr = smem_u32(sv + stage * kTileBytes);
-        const uint32_t a = tmem + kColP + (uint32_t)(j & 1) * (BN / 2);
+        const uint32_t a = tmem + kColS + (uint32_t)(j & 1) * BN;  // P lies over S
+        const uint32_t o = tmem + kColO + (uint32_t)(j & 1) * HD;  // the warpgroup's accumulator
 #pragma unroll
         for (int kk = 0; kk < BN / 16; ++kk)
-          umma_ts(tmem + kColO, a + 8u * kk,
+          umma_ts(o, a + 8u * kk,
                   smem_desc_sw128(v_addr + (uint32_t)kk * 2048u, kHalfBytes, 1024), idesc_o,
-                  (j > 0 || kk > 0) ? 1u : 0u);
+                  (j > 1 || kk > 0) ? 1u : 0u);
         umma_commit(v_empty + stage);
-        umma_commit(pv_done);
+        umma_commit(pv_done + (j & 1));
         if (j + 2 < T) issue_s(j + 2);
       }
     }
   } else if (T > 0) {
     // ------------------------------------------------------------- softmax --
     const int quad = warp & 3;               // TMEM lane quadrant this warp may touch
+    const int wg = (warp - 2) >> 2;          // warpgroup 0 takes the even key tiles, 1 the odd ones
     const int r = quad * 32 + lane;          // row of the M-tile
     const bool row_ok = r < rows_valid;
     const int nl = nl0 + r / p.group;
     const int hh = r % p.group;
     const int node = min(nl, p.NL - 1) / p.L;
     const uint32_t lane_base = (uint32_t)(quad * 32);
+    const uint32_t col_s = kColS + (uint32_t)wg * BN;  // this warpgroup's S (and P) buffer
+    const uint32_t col_o = kColO + (uint32_t)wg * HD;  // and its accumulator
     const float k2 = p.scale_log2;
     float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
-    for (int j = 0; j < T; ++j) {
-      const int buf = j & 1;
+    int mine = 0;  // tiles this warpgroup has finished
+    for (int j = wg; j < T; j += 2, ++mine) {
       // wait outcomes are made warp-uniform: the TMEM accesses below are warp-collective
-      if (!__all_sync(0xffffffffu, mbar_wait(s_full + buf, (uint32_t)(j >> 1) & 1u, abort_flag))) {
+      if (!__all_sync(0xffffffffu, mbar_wait(s_full + wg, (uint32_t)mine & 1u, abort_flag))) {
         ok = false;
         break;
       }
       tc_fence_after_sync();
       uint32_t s[BN];
-      tmem_ld_x128(tmem_addr(tmem, lane_base, kColS + (uint32_t)buf * BN), s);
+      tmem_ld_x128(tmem_addr(tmem, lane_base, col_s), s);
       // visible columns of this row in this tile: [lo, hi)
       const int t = t_begin + j;
       int lo, hi;
@@ -273,18 +284,20 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         lo = node * p.L - (kb_start + (t - p.TP) * BN);
         hi = lo + p.L;
       }
-      float mx = -INFINITY;
-      if (lo <= 0 && hi >= BN) {
+      if (!(lo <= 0 && hi >= BN)) {
 #pragma unroll
-        for (int c = 0; c < BN; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
-      } else {
-#pragma unroll
-        for (int c = 0; c < BN; ++c) {
-          const float x = (c >= lo && c < hi) ? __uint_as_float(s[c]) : -INFINITY;
-          s[c] = __float_as_uint(x);
-          mx = fmaxf(mx, x);
-        }
+        for (int c = 0; c < BN; ++c)
+          s[c] = (c >= lo && c < hi) ? s[c] : 0xff800000u;  // -inf
       }
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < BN; c += 4) {
+        mx0 = fmaxf(mx0, __uint_as_float(s[c]));
+        mx1 = fmaxf(mx1, __uint_as_float(s[c + 1]));
+        mx2 = fmaxf(mx2, __uint_as_float(s[c + 2]));
+        mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
+      }
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
       const float m_new = fmaxf(m_run, mx * k2);
       const bool need = (m_new - m_run) > kRescaleLog2;  // false when both are -inf
       if (__any_sync(0xffffffffu, need)) {
@@ -294,8 +307,9 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
           l_run *= corr;
           m_run = m_new;
         }
-        if (j > 0) {  // O holds the products of tiles 0..j-1: wait for them, then rescale
-          if (!__all_sync(0xffffffffu, mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, abort_flag))) {
+        if (mine > 0) {  // the accumulator holds this warpgroup's earlier tiles: wait, then rescale
+          if (!__all_sync(0xffffffffu,
+                          mbar_wait(pv_done + wg, (uint32_t)(mine - 1) & 1u, abort_flag))) {
             ok = false;
             break;
           }
@@ -303,73 +317,98 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
           for (int c0 = 0; c0 < HD; c0 += 32) {
             uint32_t o[32];
-            tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + c0), o);
+            tmem_ld_x32(tmem_addr(tmem, lane_base, col_o + c0), o);
 #pragma unroll
             for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * corr);
-            tmem_st_x32(tmem_addr(tmem, lane_base, kColO + c0), o);
+            tmem_st_x32(tmem_addr(tmem, lane_base, col_o + c0), o);
           }
           tmem_wait_st();
         }
       }
       const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
       uint32_t pk[BN / 2];
-      float sum0 = 0.f, sum1 = 0.f;
+      float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
 #pragma unroll
-      for (int c = 0; c < BN; c += 2) {
+      for (int c = 0; c < BN; c += 4) {
         const float p0 = ex2(fmaf(__uint_as_float(s[c]), k2, -m_use));
         const float p1 = ex2(fmaf(__uint_as_float(s[c + 1]), k2, -m_use));
-        sum0 += p0;
-        sum1 += p1;
+        const float p2 = ex2(fmaf(__uint_as_float(s[c + 2]), k2, -m_use));
+        const float p3 = ex2(fmaf(__uint_as_float(s[c + 3]), k2, -m_use));
+        sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
         pk[c >> 1] = pack_bf16(p0, p1);
+        pk[(c >> 1) + 1] = pack_bf16(p2, p3);
       }
-      l_run += sum0 + sum1;
-      tmem_st_x64(tmem_addr(tmem, lane_base, kColP + (uint32_t)buf * (BN / 2)), pk);
+      l_run += (sum0 + sum1) + (sum2 + sum3);
+      // P goes over the first half of the S columns just read (every thread owns its lane)
+      tmem_st_x64(tmem_addr(tmem, lane_base, col_s), pk);
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(p_ready + buf);
+      mbar_arrive(p_ready + wg);
     }
     // ------------------------------------------------------------ epilogue --
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(pv_done, (uint32_t)(T - 1) & 1u, abort_flag));
+    // Each warpgroup waits for its own accumulator, the two exchange their
+    // (reference maximum, sum) per row through two spare tensor-memory columns
+    // of their S buffers, and each then merges and stores one half of the
+    // columns of every row.
+    if (ok && mine > 0)
+      ok = __all_sync(0xffffffffu, mbar_wait(pv_done + wg, (uint32_t)(mine - 1) & 1u, abort_flag));
+    constexpr uint32_t kColMl = BN / 2;  // first S column that no P lies over
+    tmem_st_x2(tmem_addr(tmem, lane_base, col_s + kColMl), __float_as_uint(m_run),
+               __float_as_uint(l_run));
+    tmem_wait_st();
+    tc_fence_before_sync();
+    asm volatile("bar.sync 1, 256;" ::: "memory");  // all eight softmax warps, whatever `ok` says
+    tc_fence_after_sync();
+    uint32_t um, ul;
+    tmem_ld_x2(tmem_addr(tmem, lane_base, kColS + (uint32_t)(wg ^ 1) * BN + kColMl), um, ul);
+    const float m_o = __uint_as_float(um), l_o = __uint_as_float(ul);  // the other warpgroup's
+    const float m_a = wg == 0 ? m_run : m_o, l_a = wg == 0 ? l_run : l_o;
+    const float m_b = wg == 0 ? m_o : m_run, l_b = wg == 0 ? l_o : l_run;
+    const float m_all = fmaxf(m_a, m_b);
+    // an accumulator whose warpgroup saw no key of this row (or no tile at all) is left out
+    const bool has_a = m_a != -INFINITY, has_b = m_b != -INFINITY;
+    const float w_a = has_a ? ex2(m_a - m_all) : 0.f;
+    const float w_b = has_b ? ex2(m_b - m_all) : 0.f;
+    const float l_all = w_a * l_a + w_b * l_b;
     if (ok) {
-      tc_fence_after_sync();
-      if (p.splits == 1) {
-        const float inv = 1.0f / l_run;
-        __nv_bfloat16* dst =
-            p.out + (((int64_t)b * p.NL + nl) * p.Hq + (int64_t)g * p.group + hh) * HD;
+      const float inv = p.splits == 1 ? 1.0f / l_all : 1.0f;
+      const float f_a = w_a * inv, f_b = w_b * inv;
+      const int64_t tile = ((int64_t)split * gridDim.y + bg) * p.MT + mt;
+      __nv_bfloat16* dst =
+          p.out + (((int64_t)b * p.NL + nl) * p.Hq + (int64_t)g * p.group + hh) * HD;
+      float* po = p.part_o + (tile * BM + r) * HD;
 #pragma unroll
-        for (int c0 = 0; c0 < HD; c0 += 32) {
-          uint32_t o[32];
-          tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + c0), o);
-          if (row_ok) {
+      for (int c0 = wg * 64; c0 < wg * 64 + 64; c0 += 32) {
+        uint32_t oa[32], ob[32];
+        tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + c0), oa);
+        tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + HD + c0), ob);
+        float o[32];
+#pragma unroll
+        for (int c = 0; c < 32; ++c)
+          o[c] = (has_a ? __uint_as_float(oa[c]) * f_a : 0.f) +
+                 (has_b ? __uint_as_float(ob[c]) * f_b : 0.f);
+        if (row_ok) {
+          if (p.splits == 1) {
 #pragma unroll
             for (int c = 0; c < 32; c += 8) {
               uint4 w;
-              w.x = pack_bf16(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
-              w.y = pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
-              w.z = pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
-              w.w = pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+              w.x = pack_bf16(o[c], o[c + 1]);
+              w.y = pack_bf16(o[c + 2], o[c + 3]);
+              w.z = pack_bf16(o[c + 4], o[c + 5]);
+              w.w = pack_bf16(o[c + 6], o[c + 7]);
               *reinterpret_cast<uint4*>(dst + c0 + c) = w;
             }
-          }
-        }
-      } else {
-        const int64_t tile = ((int64_t)split * gridDim.y + bg) * p.MT + mt;
-        float* po = p.part_o + (tile * BM + r) * HD;
-        float* pml = p.part_ml + (tile * BM + r) * 2;
-#pragma unroll
-        for (int c0 = 0; c0 < HD; c0 += 32) {
-          uint32_t o[32];
-          tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + c0), o);
-          if (row_ok) {
+          } else {
 #pragma unroll
             for (int c = 0; c < 32; c += 4)
-              *reinterpret_cast<uint4*>(po + c0 + c) = make_uint4(o[c], o[c + 1], o[c + 2], o[c + 3]);
+              *reinterpret_cast<float4*>(po + c0 + c) = make_float4(o[c], o[c + 1], o[c + 2], o[c + 3]);
           }
         }
-        if (row_ok) {
-          pml[0] = m_run;
-          pml[1] = l_run;
-        }
+      }
+      if (p.splits > 1 && row_ok && wg == 0) {
+        float* pml = p.part_ml + (tile * BM + r) * 2;
+        pml[0] = m_all;
+        pml[1] = l_all;
       }
     }
   }
@@ -470,7 +509,7 @@ Plan make_plan(const spiffy_attn_desc& d) {
   // Fewer CTAs than SMs: cut the key tiles of each M-tile into slices so that
   // the context streams through more SMs at once.
   int splits = 1;
-  if (pl.tiles < 120) {
+  if (pl.tiles < 120 && pl.TP + 1 >= 8) {  // a merge pass costs about three key tiles
     splits = (int)(148 / pl.tiles);
     if (splits > pl.TP + 1) splits = pl.TP + 1;
     if (splits < 1) splits = 1;

@@ -171,6 +171,22 @@ __device__ __forceinline__ void tmem_st_x128(uint32_t taddr, const uint32_t (&r)
       : "memory");
 }
 
+// Two columns of row `lane` of the warp's TMEM quadrant.
+__device__ __forceinline__ void tmem_ld_x2(uint32_t taddr, uint32_t& r0, uint32_t& r1) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0,%1}, [%2];\n"
+      "tcgen05.wait::ld.sync.aligned;\n"
+      : "=r"(r0), "=r"(r1)
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_x2(uint32_t taddr, uint32_t r0, uint32_t r1) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1,%2};\n"
+               :
+               : "r"(taddr), "r"(r0), "r"(r1)
+               : "memory");
+}
+
 // --------------------------------------------------------------------- MMA --
 // Shared-memory matrix descriptor of a 128-byte-swizzled operand tile whose
 // 8-row (1024-byte) swizzle atoms are `sbo_bytes` apart; `lbo_bytes` is the
