@@ -189,9 +189,10 @@ spiffy_status spiffy_unmask_decide(const spiffy_decide_desc* desc,
  * spiffy_unmask_decide.  Differences:
  *   - A shape whose scratch need (spiffy_unmask_decide_workspace) exceeds
  *     SPIFFY_DECIDE_STATIC_BYTES is refused with SPIFFY_EUNSUPPORTED and nothing
- *     is launched.  The limit (512 KiB) covers every benchmark shape, the
- *     largest being B*N*L = 4096 rows; batches of several ten thousand rows
- *     go beyond it and have to use the regular entry point.
+ *     is launched.  The limit (2 MiB) covers every benchmark shape, the
+ *     largest being B*N*L = 4096 rows of a 126k vocabulary (1 MiB); batches of
+ *     ten thousand rows and more go beyond it and have to use the regular
+ *     entry point.
  *   - The first call on each device looks up the array's device address
  *     (cudaGetSymbolAddress, with that device current) and keeps it; make that
  *     first call outside any stream capture.
@@ -201,7 +202,7 @@ spiffy_status spiffy_unmask_decide(const spiffy_decide_desc* desc,
  *     from two threads without ordering) race on it and give undefined
  *     results: order them on one stream or with events.
  */
-#define SPIFFY_DECIDE_STATIC_BYTES (512u << 10)
+#define SPIFFY_DECIDE_STATIC_BYTES (2u << 20)
 spiffy_status spiffy_unmask_decide_static(const spiffy_decide_desc* desc,
                                           const void* logits,
                                           const int32_t* block_tokens,

@@ -3,7 +3,8 @@
 //
 //   decide_reduce_kernel    streams the logits rows of still-masked positions
 //                           once (the HBM-bound part): per (row, vocabulary
-//                           slice) an online (max, argmax, sum of exponentials)
+//                           slice) the maximum, the sum of exponentials and the
+//                           lowest index that attains the maximum
 //   decide_finalize_kernel  per node: merges the slices in a fixed order, turns
 //                           them into (confidence, top token) and applies the
 //                           unmasking rule of Sec. 3.1
@@ -19,7 +20,10 @@ namespace spiffy {
 namespace {
 
 constexpr int kReduceThreads = 256;
-constexpr int kUnroll = 4;
+#ifndef SPIFFY_DECIDE_UNROLL
+#define SPIFFY_DECIDE_UNROLL 4
+#endif
+constexpr int kUnroll = SPIFFY_DECIDE_UNROLL;  // 128-bit loads in flight per thread
 
 struct __align__(16) Partial {
   float m;    // slice maximum (-inf for an empty slice)
@@ -42,27 +46,7 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   return v;
 }
 
-// Running state of one thread (or of a merged group of threads).
-struct Acc {
-  float m = -INFINITY;  // running maximum
-  float ml = 0.f;       // m * log2(e), 0 while m is still -inf
-  float s = 0.f;        // sum of exp(x - m)
-  int idx = 0x7fffffff;
-};
-
-__device__ __forceinline__ void raise_max(Acc& a, float vm, int idx) {
-  const float nl = vm * kLog2e;
-  a.s *= ex2(a.ml - nl);
-  a.m = vm;
-  a.ml = nl;
-  a.idx = idx;
-}
-
-__device__ __forceinline__ float term(const Acc& a, float x) {
-  return ex2(fmaf(x, kLog2e, -a.ml));
-}
-
-// (value desc, index asc) merge of two accumulators.
+// (value desc, index asc) merge of two partial results.
 __device__ __forceinline__ void merge(float& m, float& s, int& idx, float m2,
                                       float s2, int idx2) {
   if (m2 > m || (m2 == m && idx2 < idx)) idx = idx2;
@@ -79,31 +63,39 @@ struct Elem;
 template <>
 struct Elem<__nv_bfloat16> {
   static constexpr int kPerVec = 8;
-  static __device__ __forceinline__ void consume(Acc& a, uint4 v, int base) {
+  static constexpr uint32_t kNegInf = 0xff80ff80u;  // two bf16 -inf
+  static __device__ __forceinline__ float lo(uint32_t w) { return __uint_as_float(w << 16); }
+  static __device__ __forceinline__ float hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+  static __device__ __forceinline__ __nv_bfloat162 pk(uint32_t w) {
+    return *reinterpret_cast<const __nv_bfloat162*>(&w);
+  }
+  // exact maximum of a group of vectors, on the packed bf16 pipe
+  static __device__ __forceinline__ float gmax(const uint4 (&v)[kUnroll]) {
+    __nv_bfloat162 p = __hmax2(__hmax2(pk(v[0].x), pk(v[0].y)), __hmax2(pk(v[0].z), pk(v[0].w)));
+#pragma unroll
+    for (int k = 1; k < kUnroll; ++k)
+      p = __hmax2(p, __hmax2(__hmax2(pk(v[k].x), pk(v[k].y)), __hmax2(pk(v[k].z), pk(v[k].w))));
+    return fmaxf(__low2float(p), __high2float(p));
+  }
+  // sum over the vector of 2^(x * log2e - ml)
+  static __device__ __forceinline__ float sum_terms(uint4 v, float ml) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    float f[8];
+    float t = 0.f;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      f[2 * i] = __uint_as_float(w[i] << 16);
-      f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    for (int i = 0; i < 4; ++i)
+      t += ex2(fmaf(lo(w[i]), kLog2e, -ml)) + ex2(fmaf(hi(w[i]), kLog2e, -ml));
+    return t;
+  }
+  // position of the first element equal to x, kPerVec if there is none
+  static __device__ __forceinline__ int first_equal(uint4 v, float x) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    int j = kPerVec;
+#pragma unroll
+    for (int i = 3; i >= 0; --i) {
+      j = (hi(w[i]) == x) ? 2 * i + 1 : j;
+      j = (lo(w[i]) == x) ? 2 * i : j;
     }
-    // exact maximum of the eight inputs on the packed bf16 pipe
-    __nv_bfloat162 p0 = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&w[0]),
-                                *reinterpret_cast<const __nv_bfloat162*>(&w[1]));
-    __nv_bfloat162 p1 = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&w[2]),
-                                *reinterpret_cast<const __nv_bfloat162*>(&w[3]));
-    p0 = __hmax2(p0, p1);
-    const float vm = fmaxf(__low2float(p0), __high2float(p0));
-    if (vm > a.m) {
-      int j = 7;
-#pragma unroll
-      for (int i = 6; i >= 0; --i) j = (f[i] == vm) ? i : j;
-      raise_max(a, vm, base + j);
-    }
-    float t[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) t[i] = term(a, f[i]);
-    a.s += ((t[0] + t[1]) + (t[2] + t[3])) + ((t[4] + t[5]) + (t[6] + t[7]));
+    return j;
   }
   static __device__ __forceinline__ float load1(const __nv_bfloat16* p) {
     return __bfloat162float(*p);
@@ -113,22 +105,34 @@ struct Elem<__nv_bfloat16> {
 template <>
 struct Elem<float> {
   static constexpr int kPerVec = 4;
-  static __device__ __forceinline__ void consume(Acc& a, uint4 v, int base) {
-    const float f[4] = {__uint_as_float(v.x), __uint_as_float(v.y),
-                        __uint_as_float(v.z), __uint_as_float(v.w)};
-    const float vm = fmaxf(fmaxf(f[0], f[1]), fmaxf(f[2], f[3]));
-    if (vm > a.m) {
-      int j = 3;
+  static constexpr uint32_t kNegInf = 0xff800000u;
+  static __device__ __forceinline__ float gmax(const uint4 (&v)[kUnroll]) {
+    float g = -INFINITY;
 #pragma unroll
-      for (int i = 2; i >= 0; --i) j = (f[i] == vm) ? i : j;
-      raise_max(a, vm, base + j);
-    }
-    a.s += (term(a, f[0]) + term(a, f[1])) + (term(a, f[2]) + term(a, f[3]));
+    for (int k = 0; k < kUnroll; ++k)
+      g = fmaxf(g, fmaxf(fmaxf(__uint_as_float(v[k].x), __uint_as_float(v[k].y)),
+                         fmaxf(__uint_as_float(v[k].z), __uint_as_float(v[k].w))));
+    return g;
+  }
+  static __device__ __forceinline__ float sum_terms(uint4 v, float ml) {
+    return (ex2(fmaf(__uint_as_float(v.x), kLog2e, -ml)) + ex2(fmaf(__uint_as_float(v.y), kLog2e, -ml))) +
+           (ex2(fmaf(__uint_as_float(v.z), kLog2e, -ml)) + ex2(fmaf(__uint_as_float(v.w), kLog2e, -ml)));
+  }
+  static __device__ __forceinline__ int first_equal(uint4 v, float x) {
+    int j = kPerVec;
+    j = (__uint_as_float(v.w) == x) ? 3 : j;
+    j = (__uint_as_float(v.z) == x) ? 2 : j;
+    j = (__uint_as_float(v.y) == x) ? 1 : j;
+    j = (__uint_as_float(v.x) == x) ? 0 : j;
+    return j;
   }
   static __device__ __forceinline__ float load1(const float* p) { return *p; }
 };
 
-// grid = (splits, B*N*L); one CTA reduces one vocabulary slice of one row.
+// grid = (splits, B*N*L); one CTA reduces one vocabulary slice of one row.  A
+// slice is at most kReduceThreads * kUnroll vectors, so that every thread holds
+// its whole share in registers: all loads go out at once, the slice maximum is
+// found first and the exponentials are then taken against it directly.
 template <typename T>
 __global__ void __launch_bounds__(kReduceThreads)
 decide_reduce_kernel(const T* __restrict__ logits, int64_t row_stride, int V,
@@ -144,49 +148,72 @@ decide_reduce_kernel(const T* __restrict__ logits, int64_t row_stride, int V,
   const int64_t begin = (int64_t)split * chunk;
   const int64_t end = min((int64_t)V, begin + chunk);
   constexpr int EPV = Elem<T>::kPerVec;
+  constexpr uint32_t NI = Elem<T>::kNegInf;
   const T* base = logits + (int64_t)row * row_stride;
-  Acc a;
-  if (begin < end) {
-    const int nvec = (int)((end - begin) / EPV);
-    const uint4* p = reinterpret_cast<const uint4*>(base + begin);
-    for (int i = threadIdx.x; i < nvec; i += kReduceThreads * kUnroll) {
-      uint4 v[kUnroll];
+  const int nvec = begin < end ? (int)((end - begin) / EPV) : 0;  // <= kReduceThreads * kUnroll
+  const int ntail = begin < end ? (int)(end - begin) - nvec * EPV : 0;  // < EPV, last slice only
+  const uint4* p = reinterpret_cast<const uint4*>(base + begin);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  // 1. the thread's vectors t, t + 256, ...; thread 0 also takes the ragged tail
+  uint4 v[kUnroll];
 #pragma unroll
-      for (int k = 0; k < kUnroll; ++k)
-        if (i + k * kReduceThreads < nvec) v[k] = ld_stream(p + i + k * kReduceThreads);
+  for (int u = 0; u < kUnroll; ++u)
+    v[u] = (tid + u * kReduceThreads < nvec) ? ld_stream(p + tid + u * kReduceThreads)
+                                             : make_uint4(NI, NI, NI, NI);
+  float tail[EPV];
 #pragma unroll
-      for (int k = 0; k < kUnroll; ++k)
-        if (i + k * kReduceThreads < nvec)
-          Elem<T>::consume(a, v[k], (int)begin + (i + k * kReduceThreads) * EPV);
-    }
-    // ragged tail of the slice (fewer than one vector)
-    const int64_t tail = begin + (int64_t)nvec * EPV;
-    if (threadIdx.x == 0) {
-      for (int64_t e = tail; e < end; ++e) {
-        const float x = Elem<T>::load1(base + e);
-        if (x > a.m) raise_max(a, x, (int)e);
-        a.s += term(a, x);
-      }
-    }
+  for (int e = 0; e < EPV; ++e)
+    tail[e] = (tid == 0 && e < ntail) ? Elem<T>::load1(base + begin + (int64_t)nvec * EPV + e) : -INFINITY;
+  // 2. slice maximum: lanes, warps
+  float m = Elem<T>::gmax(v);
+#pragma unroll
+  for (int e = 0; e < EPV; ++e) m = fmaxf(m, tail[e]);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+  __shared__ float warp_m[kReduceThreads / 32], warp_s[kReduceThreads / 32];
+  __shared__ int slice_idx;
+  if (lane == 0) warp_m[warp] = m;
+  if (tid == 0) slice_idx = 0x7fffffff;
+  __syncthreads();
+  m = warp_m[0];
+#pragma unroll
+  for (int w = 1; w < kReduceThreads / 32; ++w) m = fmaxf(m, warp_m[w]);
+  // 3. sum of exp(x - m) and the lowest index that attains m
+  const float ml = (m == -INFINITY) ? 0.f : m * kLog2e;  // an all -inf slice sums to 0
+  float s = 0.f;
+  int idx = 0x7fffffff;
+#pragma unroll
+  for (int u = kUnroll - 1; u >= 0; --u) {
+    s += Elem<T>::sum_terms(v[u], ml);
+    const int j = Elem<T>::first_equal(v[u], m);
+    if (j < EPV) idx = (int)begin + (tid + u * kReduceThreads) * EPV + j;  // padding never matches a finite m
   }
-  // CTA-wide merge in a fixed order: lanes, then warps
-  float m = a.m, s = a.s;
-  int idx = a.idx;
+  if (ntail > 0 && tid == 0) {
+    int tidx = 0x7fffffff;
+#pragma unroll
+    for (int e = EPV - 1; e >= 0; --e) {
+      s += ex2(fmaf(tail[e], kLog2e, -ml));  // -inf beyond the tail: adds 0
+      if (e < ntail && tail[e] == m) tidx = (int)begin + nvec * EPV + e;
+    }
+    idx = min(idx, tidx);
+  }
+  if (m == -INFINITY) idx = 0x7fffffff;
+  // fixed order: lanes (butterfly), then warps
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
-    const float m2 = __shfl_down_sync(0xffffffffu, m, off);
-    const float s2 = __shfl_down_sync(0xffffffffu, s, off);
-    const int i2 = __shfl_down_sync(0xffffffffu, idx, off);
-    merge(m, s, idx, m2, s2, i2);
+    s += __shfl_xor_sync(0xffffffffu, s, off);
+    idx = min(idx, __shfl_xor_sync(0xffffffffu, idx, off));
   }
-  __shared__ Partial warp_part[kReduceThreads / 32];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (lane == 0) warp_part[warp] = Partial{m, s, idx, 0};
+  if (lane == 0) {
+    warp_s[warp] = s;
+    if (idx != 0x7fffffff) atomicMin(&slice_idx, idx);
+  }
   __syncthreads();
-  if (threadIdx.x == 0) {
-    for (int w = 1; w < kReduceThreads / 32; ++w)
-      merge(m, s, idx, warp_part[w].m, warp_part[w].s, warp_part[w].idx);
-    partials[(int64_t)row * splits + split] = Partial{m, s, idx, 0};
+  if (tid == 0) {
+    s = warp_s[0];
+    for (int w = 1; w < kReduceThreads / 32; ++w) s += warp_s[w];
+    partials[(int64_t)row * splits + split] = Partial{m, s, slice_idx, 0};
   }
 }
 
@@ -259,20 +286,13 @@ decide_finalize_kernel(const Partial* __restrict__ partials, int splits, int N,
 }  // namespace
 
 int decide_splits(const spiffy_decide_desc& d, int64_t* chunk_elems) {
-  // Enough CTAs to keep every SM streaming (about 8 CTAs of 256 threads per
-  // SM over 148 SMs), slices never shorter than 4096 elements and cut on
-  // 2048-element boundaries so that every slice starts on a 16-byte boundary.
-  const int64_t rows = (int64_t)d.batch * d.n_nodes * d.block_len;
-  int64_t want = (148 * 8 + rows - 1) / rows;
-  const int64_t max_by_len = (d.vocab + 4095) / 4096;
-  if (want > max_by_len) want = max_by_len;
-  if (want < 1) want = 1;
-  if (want > 64) want = 64;
-  int64_t chunk = (d.vocab + want - 1) / want;
-  chunk = (chunk + 2047) / 2048 * 2048;
-  const int splits = (int)((d.vocab + chunk - 1) / chunk);
+  // A slice is what one CTA holds in registers: kReduceThreads * kUnroll vectors
+  // of 16 bytes (8192 bf16 or 4096 fp32 logits); slices start on 16-byte boundaries.
+  const int64_t epv = d.logits_dtype == SPIFFY_BF16 ? 8 : 4;
+  const int64_t chunk = (int64_t)kReduceThreads * kUnroll * epv;
+  const int64_t splits = (d.vocab + chunk - 1) / chunk;
   if (chunk_elems) *chunk_elems = chunk;
-  return splits < 1 ? 1 : splits;
+  return (int)(splits < 1 ? 1 : splits);
 }
 
 size_t decide_workspace_bytes(const spiffy_decide_desc& d) {

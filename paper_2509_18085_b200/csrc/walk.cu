@@ -35,10 +35,19 @@ accept_walk_kernel(int N, int L, const int32_t* __restrict__ block_tokens,
     int32_t* s_top = s_state + N * L;
     int32_t* s_off = s_top + N * L;
     int32_t* s_idx = s_off + (N + 1);
-    for (int i = lane; i < N * L; i += 32) { s_state[i] = state[i]; s_top[i] = top[i]; }
-    for (int i = lane; i <= N; i += 32) s_off[i] = off[i];
-    for (int i = lane; i < parent_cap; i += 32) s_idx[i] = idx[i];
-    for (int i = lane; i < N; i += 32) s_bits[i] = ubits[i];
+    // asynchronous copies: every load is in flight before the first one is waited for
+    auto copy4 = [](void* dst, const void* src) {
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(
+                       (uint32_t)__cvta_generic_to_shared(dst)),
+                   "l"(src)
+                   : "memory");
+    };
+    for (int i = lane; i < N * L; i += 32) { copy4(s_state + i, state + i); copy4(s_top + i, top + i); }
+    for (int i = lane; i <= N; i += 32) copy4(s_off + i, off + i);
+    for (int i = lane; i < parent_cap; i += 32) copy4(s_idx + i, idx + i);
+    for (int i = lane; i < 2 * N; i += 32)
+      copy4(reinterpret_cast<int32_t*>(s_bits) + i, reinterpret_cast<const int32_t*>(ubits) + i);
+    asm volatile("cp.async.wait_all;" ::: "memory");
     __syncwarp();
     state = s_state; top = s_top; off = s_off; idx = s_idx; ubits = s_bits;
   }

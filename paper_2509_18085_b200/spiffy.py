@@ -29,7 +29,7 @@ EXPORTS = (
     "spiffy_accept_walk", "spiffy_status_string", "spiffy_launch_count",
     "spiffy_unmask_decide_static",
 )
-DECIDE_STATIC_BYTES = 512 << 10
+DECIDE_STATIC_BYTES = 2 << 20
 
 
 class SpiffyError(RuntimeError):
