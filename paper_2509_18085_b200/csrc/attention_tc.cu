@@ -44,8 +44,7 @@ using namespace sm100;
 constexpr int BM = 128;       // rows of an M-tile (TMEM lanes)
 constexpr int BN = 128;       // keys per key tile
 constexpr int HD = 128;       // head dimension
-constexpr int KS = 3;         // K ring stages
-constexpr int VS = 3;         // V ring stages
+constexpr int kMaxStages = 3;  // most stages a K or V ring has
 constexpr int kThreads = 320;  // producer warp, MMA warp, two softmax warpgroups
 constexpr int kHalfBytes = BN * 128;           // one 64-column half of a tile: 128 rows x 128 B
 constexpr int kTileBytes = 2 * kHalfBytes;     // 32 KB
@@ -55,17 +54,22 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;
 constexpr float kRescaleLog2 = 8.0f;
 
+// NQ M-tiles per CTA: NQ Q tiles, a K ring of 3 stages and a V ring of 4 - NQ
+// stages: 7 tiles of 32 KB either way.
+template <int NQ>
 struct Smem {
+  static constexpr int ks = 3, vs = 4 - NQ;
   static constexpr int q = 0;
-  static constexpr int k = q + kTileBytes;
-  static constexpr int v = k + KS * kTileBytes;
-  static constexpr int bars = v + VS * kTileBytes;
-  static constexpr int n_bars = 1 + 2 * KS + 2 * VS + 2 + 2 + 2;
+  static constexpr int k = q + NQ * kTileBytes;
+  static constexpr int v = k + ks * kTileBytes;
+  static constexpr int bars = v + vs * kTileBytes;
+  static constexpr int n_bars = 1 + 4 * kMaxStages + 2 + 2 + 2;
   static constexpr int tmem = bars + 8 * n_bars;
   static constexpr int abort_flag = tmem + 8;
   static constexpr int total = abort_flag + 8;
 };
-constexpr int kSmemBytes = Smem::total + 1024;  // slack for 1024-byte alignment
+constexpr int kSmemBytes = Smem<1>::total + 1024;  // slack for 1024-byte alignment
+static_assert(Smem<1>::total == Smem<2>::total, "both layouts use the same amount");
 
 struct Params {
   int B, N, L, P, Hq, Hkv, group;
@@ -99,6 +103,11 @@ __device__ __forceinline__ void mbar_wait_quiet(uint64_t* bar, uint32_t parity) 
     if (mbar_try_wait(bar, parity)) return;
 }
 
+// NQ = 1: the CTA owns one M-tile and its two softmax warpgroups alternate over
+// the key tiles.  NQ = 2: the CTA owns two neighbouring M-tiles, one per
+// warpgroup, and every K/V tile brought into shared memory serves both, which
+// halves the L2-to-SM traffic per flop.
+template <int NQ>
 __global__ void __launch_bounds__(kThreads, 1)
 graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                           const __grid_constant__ CUtensorMap tm_kp,
@@ -108,10 +117,12 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-  uint8_t* sq = smem + Smem::q;
-  uint8_t* sk = smem + Smem::k;
-  uint8_t* sv = smem + Smem::v;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Smem::bars);
+  using SM = Smem<NQ>;
+  constexpr int KS = SM::ks, VS = SM::vs;
+  uint8_t* sq = smem + SM::q;
+  uint8_t* sk = smem + SM::k;
+  uint8_t* sv = smem + SM::v;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::bars);
   uint64_t* q_full = bars;
   uint64_t* k_full = bars + 1;
   uint64_t* k_empty = k_full + KS;
@@ -120,20 +131,19 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
   uint64_t* s_full = v_empty + VS;   // [2]
   uint64_t* p_ready = s_full + 2;    // [2]
   uint64_t* pv_done = p_ready + 2;   // [2], one per softmax warpgroup
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + Smem::tmem);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + Smem::abort_flag);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + SM::tmem);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SM::abort_flag);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int mt = blockIdx.x;
+  const int mt = blockIdx.x * NQ;  // first M-tile of this CTA
   const int bg = blockIdx.y;
   const int b = bg / p.Hkv, g = bg % p.Hkv;
   const int split = blockIdx.z;
 
   // this CTA's rows and key tiles
   const int nl0 = mt * p.TNL;
-  const int nl_count = min(p.TNL, p.NL - nl0);
-  const int rows_box = p.TNL * p.group;        // rows the Q box writes
-  const int rows_valid = nl_count * p.group;   // rows that exist
+  const int nl_count = min(NQ * p.TNL, p.NL - nl0);  // over all M-tiles of the CTA
+  const int rows_box = p.TNL * p.group;        // rows one Q box writes
   const int n_lo = nl0 / p.L, n_hi = (nl0 + nl_count - 1) / p.L;
   const int kb_start = n_lo * p.L;
   const int TB = ((n_hi - n_lo + 1) * p.L + BN - 1) / BN;
@@ -155,8 +165,8 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
   // rows of the Q tile that the TMA box does not write must be finite
   for (int i = rows_box * 8 + threadIdx.x; i < BM * 8; i += kThreads) {
     const uint4 z = make_uint4(0, 0, 0, 0);
-    reinterpret_cast<uint4*>(sq)[i] = z;
-    reinterpret_cast<uint4*>(sq + kHalfBytes)[i] = z;
+#pragma unroll
+    for (int h = 0; h < 2 * NQ; ++h) reinterpret_cast<uint4*>(sq + h * kHalfBytes)[i] = z;
   }
   fence_proxy_async_smem();
   if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
@@ -172,9 +182,13 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     if (lane == 0 && T > 0) {
       prefetch_tensormap(&tm_q);
       prefetch_tensormap(p.TP > 0 ? &tm_kp : &tm_kb);
-      mbar_arrive_expect_tx(q_full, 2u * rows_box * 128u);
-      tma_load_4d(sq, &tm_q, q_full, 0, g * p.group, nl0, b);
-      tma_load_4d(sq + kHalfBytes, &tm_q, q_full, 64, g * p.group, nl0, b);
+      mbar_arrive_expect_tx(q_full, (uint32_t)NQ * 2u * rows_box * 128u);
+#pragma unroll
+      for (int q = 0; q < NQ; ++q) {  // an M-tile beyond the last one reads as zeros
+        tma_load_4d(sq + q * kTileBytes, &tm_q, q_full, 0, g * p.group, nl0 + q * p.TNL, b);
+        tma_load_4d(sq + q * kTileBytes + kHalfBytes, &tm_q, q_full, 64, g * p.group,
+                    nl0 + q * p.TNL, b);
+      }
       int issued_k = 0, issued_v = 0;
       bool ok = true;
       auto load = [&](bool is_k, int j) {
@@ -212,50 +226,88 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     if (lane == 0 && T > 0) {
       constexpr uint32_t idesc_s = idesc_bf16_f32(BM, BN, false, false);
       constexpr uint32_t idesc_o = idesc_bf16_f32(BM, HD, false, true);
-      const uint32_t q_addr = smem_u32(sq);
       bool ok = mbar_wait(q_full, 0, abort_flag);
-      auto issue_s = [&](int j) {
-        const int stage = j % KS;
-        if (!mbar_wait(k_full + stage, (uint32_t)(j / KS) & 1u, abort_flag)) { ok = false; return; }
-        tc_fence_after_sync();
-        const uint32_t k_addr = smem_u32(sk + stage * kTileBytes);
-        const uint32_t d = tmem + kColS + (uint32_t)(j & 1) * BN;
+      // S = Q K^T of key tile j into S buffer `buf`, from Q tile `qt`
+      auto issue_s = [&](int j, int buf, int qt) {
+        const uint32_t q_addr = smem_u32(sq + qt * kTileBytes);
+        const uint32_t k_addr = smem_u32(sk + (j % KS) * kTileBytes);
+        const uint32_t d = tmem + kColS + (uint32_t)buf * BN;
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk) {
           const uint32_t off = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
           umma_ss(d, smem_desc_sw128(q_addr + off, 16, 1024),
                   smem_desc_sw128(k_addr + off, 16, 1024), idesc_s, kk > 0);
         }
-        umma_commit(k_empty + stage);
-        umma_commit(s_full + (j & 1));
+        umma_commit(s_full + buf);
       };
-      if (ok) issue_s(0);
-      if (ok && T > 1) issue_s(1);
-      for (int j = 0; j < T && ok; ++j) {
-        const int stage = j % VS;
-        if (!mbar_wait(p_ready + (j & 1), (uint32_t)(j >> 1) & 1u, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(v_full + stage, (uint32_t)(j / VS) & 1u, abort_flag)) { ok = false; break; }
-        tc_fence_after_sync();
-        const uint32_t v_addr = smem_u32(sv + stage * kTileBytes);
-        const uint32_t a = tmem + kColS + (uint32_t)(j & 1) * BN;  // P lies over S
-        const uint32_t o = tmem + kColO + (uint32_t)(j & 1) * HD;  // the warpgroup's accumulator
+      // O[buf] (+)= P[buf] V of key tile j; `first` starts the accumulator
+      auto issue_pv = [&](int j, int buf, bool first) {
+        const uint32_t v_addr = smem_u32(sv + (j % VS) * kTileBytes);
+        const uint32_t a = tmem + kColS + (uint32_t)buf * BN;  // P lies over S
+        const uint32_t o = tmem + kColO + (uint32_t)buf * HD;
 #pragma unroll
         for (int kk = 0; kk < BN / 16; ++kk)
           umma_ts(o, a + 8u * kk,
                   smem_desc_sw128(v_addr + (uint32_t)kk * 2048u, kHalfBytes, 1024), idesc_o,
-                  (j > 1 || kk > 0) ? 1u : 0u);
-        umma_commit(v_empty + stage);
-        umma_commit(pv_done + (j & 1));
-        if (j + 2 < T) issue_s(j + 2);
+                  (!first || kk > 0) ? 1u : 0u);
+        umma_commit(pv_done + buf);
+      };
+      auto wait_k = [&](int j) {
+        if (ok && !mbar_wait(k_full + j % KS, (uint32_t)(j / KS) & 1u, abort_flag)) ok = false;
+        tc_fence_after_sync();
+      };
+      if constexpr (NQ == 1) {
+        // the two S buffers hold consecutive key tiles
+        auto s_tile = [&](int j) {
+          wait_k(j);
+          if (!ok) return;
+          issue_s(j, j & 1, 0);
+          umma_commit(k_empty + j % KS);
+        };
+        s_tile(0);
+        if (T > 1) s_tile(1);
+        for (int j = 0; j < T && ok; ++j) {
+          if (!mbar_wait(p_ready + (j & 1), (uint32_t)(j >> 1) & 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(v_full + j % VS, (uint32_t)(j / VS) & 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after_sync();
+          issue_pv(j, j & 1, j < 2);
+          umma_commit(v_empty + j % VS);
+          if (j + 2 < T) s_tile(j + 2);
+        }
+      } else {
+        // S buffer q belongs to M-tile q; a key tile serves both before it is released
+        wait_k(0);
+        if (ok) {
+          issue_s(0, 0, 0);
+          issue_s(0, 1, 1);
+          umma_commit(k_empty + 0);
+        }
+        for (int j = 0; j < T && ok; ++j) {
+          if (!mbar_wait(v_full + j % VS, (uint32_t)(j / VS) & 1u, abort_flag)) { ok = false; break; }
+          if (j + 1 < T) wait_k(j + 1);
+          for (int q = 0; q < 2 && ok; ++q) {
+            if (!mbar_wait(p_ready + q, (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            issue_pv(j, q, j == 0);
+            if (j + 1 < T) issue_s(j + 1, q, q);  // after PV: P of this tile has been consumed
+          }
+          if (!ok) break;
+          umma_commit(v_empty + j % VS);
+          if (j + 1 < T) umma_commit(k_empty + (j + 1) % KS);
+        }
       }
     }
   } else if (T > 0) {
     // ------------------------------------------------------------- softmax --
     const int quad = warp & 3;               // TMEM lane quadrant this warp may touch
-    const int wg = (warp - 2) >> 2;          // warpgroup 0 takes the even key tiles, 1 the odd ones
+    // NQ = 1: warpgroup 0 takes the even key tiles, 1 the odd ones, same rows;
+    // NQ = 2: warpgroup q takes every key tile for the rows of M-tile q
+    const int wg = (warp - 2) >> 2;
     const int r = quad * 32 + lane;          // row of the M-tile
+    const int nl_tile = nl0 + (NQ == 2 ? wg * p.TNL : 0);  // first (node, position) of the rows
+    const int rows_valid = max(0, min(p.TNL, p.NL - nl_tile)) * p.group;
     const bool row_ok = r < rows_valid;
-    const int nl = nl0 + r / p.group;
+    const int nl = nl_tile + r / p.group;
     const int hh = r % p.group;
     const int node = min(nl, p.NL - 1) / p.L;
     const uint32_t lane_base = (uint32_t)(quad * 32);
@@ -265,7 +317,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
     int mine = 0;  // tiles this warpgroup has finished
-    for (int j = wg; j < T; j += 2, ++mine) {
+    for (int j = (NQ == 1 ? wg : 0); j < T; j += (NQ == 1 ? 2 : 1), ++mine) {
       // wait outcomes are made warp-uniform: the TMEM accesses below are warp-collective
       if (!__all_sync(0xffffffffu, mbar_wait(s_full + wg, (uint32_t)mine & 1u, abort_flag))) {
         ok = false;
@@ -352,6 +404,44 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     // columns of every row.
     if (ok && mine > 0)
       ok = __all_sync(0xffffffffu, mbar_wait(pv_done + wg, (uint32_t)(mine - 1) & 1u, abort_flag));
+    if constexpr (NQ == 2) {
+      // each warpgroup owns its rows outright: normalise (or hand on the partial) and store
+      if (ok) {
+        tc_fence_after_sync();
+        const float inv = p.splits == 1 ? 1.0f / l_run : 1.0f;
+        const int64_t tile = ((int64_t)split * gridDim.y + bg) * p.MT + mt + wg;
+        __nv_bfloat16* dst =
+            p.out + (((int64_t)b * p.NL + nl) * p.Hq + (int64_t)g * p.group + hh) * HD;
+        float* po = p.part_o + (tile * BM + r) * HD;
+#pragma unroll
+        for (int c0 = 0; c0 < HD; c0 += 32) {
+          uint32_t o[32];
+          tmem_ld_x32(tmem_addr(tmem, lane_base, col_o + c0), o);
+          if (row_ok) {
+            if (p.splits == 1) {
+#pragma unroll
+              for (int c = 0; c < 32; c += 8) {
+                uint4 w;
+                w.x = pack_bf16(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
+                w.y = pack_bf16(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+                w.z = pack_bf16(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+                w.w = pack_bf16(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+                *reinterpret_cast<uint4*>(dst + c0 + c) = w;
+              }
+            } else {
+#pragma unroll
+              for (int c = 0; c < 32; c += 4)
+                *reinterpret_cast<uint4*>(po + c0 + c) = make_uint4(o[c], o[c + 1], o[c + 2], o[c + 3]);
+            }
+          }
+        }
+        if (p.splits > 1 && row_ok) {
+          float* pml = p.part_ml + (tile * BM + r) * 2;
+          pml[0] = m_run;
+          pml[1] = l_run;
+        }
+      }
+    } else {
     constexpr uint32_t kColMl = BN / 2;  // first S column that no P lies over
     tmem_st_x2(tmem_addr(tmem, lane_base, col_s + kColMl), __float_as_uint(m_run),
                __float_as_uint(l_run));
@@ -411,6 +501,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         pml[1] = l_all;
       }
     }
+    }  // NQ == 1
   }
 
   tc_fence_before_sync();
@@ -495,6 +586,7 @@ bool make_map(CUtensorMap* m, const void* base, int heads, int64_t rows, int out
 
 struct Plan {
   int group, TNL, NL, MT, TP, splits;
+  int nq;  // M-tiles per CTA
   int64_t tiles;  // B * Hkv * MT
 };
 
@@ -506,6 +598,9 @@ Plan make_plan(const spiffy_attn_desc& d) {
   pl.MT = (pl.NL + pl.TNL - 1) / pl.TNL;
   pl.TP = (d.prefix_len + BN - 1) / BN;
   pl.tiles = (int64_t)d.batch * d.n_kv_heads * pl.MT;
+  // Two M-tiles per CTA once the paired CTAs still fill the machine: every K/V
+  // tile then serves twice as many rows per trip from L2.
+  pl.nq = ((int64_t)d.batch * d.n_kv_heads * ((pl.MT + 1) / 2) >= 148) ? 2 : 1;
   // Fewer CTAs than SMs: cut the key tiles of each M-tile into slices so that
   // the context streams through more SMs at once.
   int splits = 1;
@@ -562,12 +657,15 @@ spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q, cons
   p.part_ml = p.part_o ? p.part_o + (size_t)pl.splits * pl.tiles * BM * HD : nullptr;
   p.status = dev_status;
 
-  if (cudaFuncSetAttribute(graph_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           kSmemBytes) != cudaSuccess)
+  if (cudaFuncSetAttribute(graph_attention_tc_kernel<1>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(graph_attention_tc_kernel<2>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
     return SPIFFY_ECUDA;
-  const dim3 grid(pl.MT, d.batch * d.n_kv_heads, pl.splits);
-  if (launch_pdl(graph_attention_tc_kernel, grid, dim3(kThreads), (size_t)kSmemBytes, stream, tm_q,
-                 tm_kp, tm_vp, tm_kb, tm_vb, p) != cudaSuccess)
+  const dim3 grid((pl.MT + pl.nq - 1) / pl.nq, d.batch * d.n_kv_heads, pl.splits);
+  auto kern = pl.nq == 2 ? graph_attention_tc_kernel<2> : graph_attention_tc_kernel<1>;
+  if (launch_pdl(kern, grid, dim3(kThreads), (size_t)kSmemBytes, stream, tm_q, tm_kp, tm_vp, tm_kb,
+                 tm_vb, p) != cudaSuccess)
     return SPIFFY_ECUDA;
   count_launch();
   if (pl.splits > 1) {
