@@ -52,6 +52,10 @@ def parse():
     ap.add_argument("--nodes", type=int, default=None, help="node count for configuration 5")
     ap.add_argument("--attn-kernel", default="auto", choices=["auto", "simt", "tcgen05"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--part", default="step", choices=["step", "attention", "decide"],
+                    help="time one library call alone on any configuration (for profiling); "
+                         "the benchmark line itself is --part step")
+    ap.add_argument("--sets", type=int, default=0, help="rotating input sets for --part (0 = enough to exceed L2)")
     return ap.parse_args()
 
 
@@ -212,10 +216,71 @@ def run_reference(args):
         "gpu_launches": 0}))
 
 
+def run_part(args):
+    """One library call alone: graph replay over rotating input sets, CUDA events.
+    Prints its own small JSON line; used for profiling the other configurations."""
+    import numpy as np
+    import torch
+    from paper_2509_18085_b200 import spiffy
+    from paper_2509_18085_b200 import workloads as W
+    from paper_2509_18085_b200.step import VerifyStep, inputs_from_workload
+
+    torch.cuda.set_device(0)
+    cfg = W.config(args.config, args.nodes)
+    attn = args.part == "attention"
+    probe = W.make(cfg, W.seed_for(args.config, 100), attention=attn, decision=not attn)
+    masked = int((probe.block_tokens == cfg.mask_id).sum())
+    attn_bytes, decide_bytes, attn_flops = algorithmic_bytes(cfg, masked)
+    per_set = attn_bytes if attn else decide_bytes
+    n_sets = args.sets or max(2, min(16, int(300e6 // per_set) + 1))
+    work = [probe] + [W.make(cfg, W.seed_for(args.config, 100 + i), attention=attn, decision=not attn)
+                      for i in range(1, n_sets)]
+    sets = [inputs_from_workload(w) for w in work]
+    kernel = {"auto": spiffy.ATTN_AUTO, "simt": spiffy.ATTN_SIMT, "tcgen05": spiffy.ATTN_TCGEN05}[args.attn_kernel]
+    step = VerifyStep(cfg, attn_kernel=kernel)
+    call = step.attention if attn else step.decide
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for x in sets:
+            call(x)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for x in sets:
+                call(x)
+        for _ in range(max(3, args.warmup // n_sets)):
+            g.replay()
+        stream.synchronize()
+        reps = max(1, args.steps // n_sets)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        e1.record(stream)
+        stream.synchronize()
+        sec = e0.elapsed_time(e1) * 1e-3 / (reps * n_sets)
+    peaks = measured_peaks()
+    masked_all = float(np.mean([(w.block_tokens == cfg.mask_id).sum() for w in work]))
+    out = {"part": args.part, "config": f"config{args.config}-{cfg.name}", "n_nodes": cfg.n_nodes,
+           "us_per_call": sec * 1e6, "input_sets": n_sets, "calls_timed": reps * n_sets}
+    if attn:
+        out.update(tflops=attn_flops / sec / 1e12, frac_of_bf16_peak=attn_flops / sec / 1e12 / peaks["bf16_tflops"],
+                   gbs=attn_bytes / sec / 1e9, frac_of_hbm=attn_bytes / sec / 1e9 / peaks["hbm_gbs"],
+                   algorithmic_flops=attn_flops, algorithmic_bytes=attn_bytes)
+    else:
+        by = algorithmic_bytes(cfg, masked_all)[1]
+        out.update(gbs=by / sec / 1e9, frac_of_hbm=by / sec / 1e9 / peaks["hbm_gbs"], algorithmic_bytes=by,
+                   masked_rows=masked_all)
+    out["peaks"] = peaks["source"]
+    print(json.dumps(out))
+
+
 def main():
     args = parse()
     if args.impl == "reference":
         return run_reference(args)
+    if args.part != "step":
+        return run_part(args)
 
     import numpy as np
     import torch
