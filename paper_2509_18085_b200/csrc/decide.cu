@@ -69,7 +69,11 @@ struct Elem<__nv_bfloat16> {
   static __device__ __forceinline__ __nv_bfloat162 pk(uint32_t w) {
     return *reinterpret_cast<const __nv_bfloat162*>(&w);
   }
-  // exact maximum of a group of vectors, on the packed bf16 pipe
+  // exact maximum of one vector / of a group of vectors, on the packed bf16 pipe
+  static __device__ __forceinline__ float vmax(uint4 v) {
+    const __nv_bfloat162 p = __hmax2(__hmax2(pk(v.x), pk(v.y)), __hmax2(pk(v.z), pk(v.w)));
+    return fmaxf(__low2float(p), __high2float(p));
+  }
   static __device__ __forceinline__ float gmax(const uint4 (&v)[kUnroll]) {
     __nv_bfloat162 p = __hmax2(__hmax2(pk(v[0].x), pk(v[0].y)), __hmax2(pk(v[0].z), pk(v[0].w)));
 #pragma unroll
@@ -106,6 +110,10 @@ template <>
 struct Elem<float> {
   static constexpr int kPerVec = 4;
   static constexpr uint32_t kNegInf = 0xff800000u;
+  static __device__ __forceinline__ float vmax(uint4 v) {
+    return fmaxf(fmaxf(__uint_as_float(v.x), __uint_as_float(v.y)),
+                 fmaxf(__uint_as_float(v.z), __uint_as_float(v.w)));
+  }
   static __device__ __forceinline__ float gmax(const uint4 (&v)[kUnroll]) {
     float g = -INFINITY;
 #pragma unroll
@@ -186,8 +194,8 @@ decide_reduce_kernel(const T* __restrict__ logits, int64_t row_stride, int V,
 #pragma unroll
   for (int u = kUnroll - 1; u >= 0; --u) {
     s += Elem<T>::sum_terms(v[u], ml);
-    const int j = Elem<T>::first_equal(v[u], m);
-    if (j < EPV) idx = (int)begin + (tid + u * kReduceThreads) * EPV + j;  // padding never matches a finite m
+    if (Elem<T>::vmax(v[u]) == m)  // rare: only the vectors that hold the slice maximum are searched
+      idx = (int)begin + (tid + u * kReduceThreads) * EPV + Elem<T>::first_equal(v[u], m);
   }
   if (ntail > 0 && tid == 0) {
     int tidx = 0x7fffffff;
