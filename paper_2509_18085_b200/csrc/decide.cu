@@ -225,8 +225,10 @@ decide_reduce_kernel(const T* __restrict__ logits, int64_t row_stride, int V,
   }
 }
 
-// grid = B*N nodes, 64 threads: thread l owns position l of the node.
-__global__ void __launch_bounds__(64)
+// grid = B*N nodes, 512 threads: eight threads per position merge the slices of
+// its row, then threads 0..63 apply the rule (thread l owns position l).
+constexpr int kFinalizeThreads = 512;
+__global__ void __launch_bounds__(kFinalizeThreads)
 decide_finalize_kernel(const Partial* __restrict__ partials, int splits, int N,
                        int L, const int32_t* __restrict__ block_tokens,
                        int mask_id, int rule, int top_s, float tau,
@@ -238,34 +240,49 @@ decide_finalize_kernel(const Partial* __restrict__ partials, int splits, int N,
   cudaGridDependencySynchronize();  // the reduce kernel's partials are visible
 #endif
   const int node = blockIdx.x;
-  const int l = threadIdx.x;
+  const int pos = threadIdx.x >> 3, sub = threadIdx.x & 7;
   __shared__ float sconf[64];
   __shared__ uint32_t sballot[2];
-  bool masked = false;
-  float conf = -INFINITY;
-  if (l < L) {
-    const int row = node * L + l;
+  if (threadIdx.x < 64) sconf[threadIdx.x] = -INFINITY;
+  __syncthreads();
+  {
+    const int row = node * L + min(pos, L - 1);
+    // the token and the partials are read together (one trip to memory); the
+    // partials of an unmasked row were never written and are ignored below
     const int32_t state = block_tokens[row];
-    int tok = state;
-    masked = state == mask_id;
-    if (masked) {
-      const Partial* p = partials + (int64_t)row * splits;
-      float m = p[0].m, s = p[0].s;
-      int idx = p[0].idx;
-      for (int k = 1; k < splits; ++k) merge(m, s, idx, p[k].m, p[k].s, p[k].idx);
-      conf = 1.0f / s;
-      tok = idx;
-      // a usable row has a finite maximum and a finite, positive sum
-      if (!(fabsf(m) < INFINITY) || !(s >= 1.0f) || !(s < INFINITY)) {
+    float m = -INFINITY, s = 0.f;
+    int idx = 0x7fffffff;
+    const Partial* p = partials + (int64_t)row * splits;
+    for (int k = sub; k < splits; k += 8) {
+      const Partial q = p[k];
+      merge(m, s, idx, q.m, q.s, q.idx);
+    }
+#pragma unroll
+    for (int off = 4; off > 0; off >>= 1) {  // fixed order inside the group of eight
+      const float m2 = __shfl_xor_sync(0xffffffffu, m, off);
+      const float s2 = __shfl_xor_sync(0xffffffffu, s, off);
+      const int i2 = __shfl_xor_sync(0xffffffffu, idx, off);
+      merge(m, s, idx, m2, s2, i2);
+    }
+    if (sub == 0 && pos < L) {
+      const bool masked = state == mask_id;
+      const float conf = masked ? 1.0f / s : -INFINITY;
+      conf_out[row] = conf;
+      tok_out[row] = masked ? idx : state;
+      sconf[pos] = conf;
+      // a usable row has a finite maximum and a finite sum of at least one
+      if (masked && (!(fabsf(m) < INFINITY) || !(s >= 1.0f) || !(s < INFINITY))) {
         if (dev_status) atomicOr(dev_status + node / N, SPIFFY_DEV_NONFINITE);
       }
     }
-    conf_out[row] = conf;
-    tok_out[row] = tok;
   }
-  sconf[l] = masked ? conf : -INFINITY;
   __syncthreads();
-  // rank among the masked positions by (confidence desc, position asc)
+  if (threadIdx.x >= 64) return;
+  const int l = threadIdx.x;
+  const bool masked = l < L && block_tokens[node * L + min(l, L - 1)] == mask_id;
+  const float conf = masked ? sconf[l] : -INFINITY;
+  // rank among the masked positions by (confidence desc, position asc); the
+  // confidence of an unmasked position is -inf and a masked one's is not
   int rank = 0;
   if (masked) {
     for (int j = 0; j < L; ++j) {
@@ -278,12 +295,16 @@ decide_finalize_kernel(const Partial* __restrict__ partials, int splits, int N,
     take = masked && rank < top_s;
   } else {
     const bool pass = masked && conf > tau;  // strict, Sec. 3.1
-    const int any = __syncthreads_or(pass ? 1 : 0);
+    const uint32_t any0 = __ballot_sync(0xffffffffu, pass);
+    if ((l & 31) == 0) sballot[l >> 5] = any0;
+    asm volatile("bar.sync 1, 64;" ::: "memory");
+    const bool any = (sballot[0] | sballot[1]) != 0u;
+    asm volatile("bar.sync 1, 64;" ::: "memory");
     take = any ? pass : (masked && rank == 0);
   }
-  const uint32_t b = __ballot_sync(0xffffffffu, take);
-  if ((l & 31) == 0) sballot[l >> 5] = b;
-  __syncthreads();
+  const uint32_t bal = __ballot_sync(0xffffffffu, take);
+  if ((l & 31) == 0) sballot[l >> 5] = bal;
+  asm volatile("bar.sync 1, 64;" ::: "memory");
   if (l == 0) {
     const uint64_t bits = (uint64_t)sballot[0] | ((uint64_t)sballot[1] << 32);
     bits_out[node] = bits;
@@ -333,7 +354,7 @@ spiffy_status launch_decide(const spiffy_decide_desc& d, const void* logits,
   // The finalize kernel's launch overlaps the tail of the reduce kernel; it
   // waits on the device (cudaGridDependencySynchronize) for the partials.
   const Partial* cpart = partials;
-  e = launch_pdl(decide_finalize_kernel, dim3(d.batch * d.n_nodes), dim3(64), (size_t)0, stream,
+  e = launch_pdl(decide_finalize_kernel, dim3(d.batch * d.n_nodes), dim3(kFinalizeThreads), (size_t)0, stream,
                  cpart, splits, (int)d.n_nodes, (int)d.block_len, block_tokens,
                  (int)d.mask_token_id, (int)d.rule, (int)d.top_s, d.threshold, conf, top_tok,
                  unmask_bits, n_unmask, dev_status);
