@@ -21,7 +21,7 @@ namespace {
 
 constexpr int kReduceThreads = 256;
 #ifndef SPIFFY_DECIDE_UNROLL
-#define SPIFFY_DECIDE_UNROLL 4
+#define SPIFFY_DECIDE_UNROLL 8
 #endif
 constexpr int kUnroll = SPIFFY_DECIDE_UNROLL;  // 128-bit loads in flight per thread
 
@@ -315,11 +315,15 @@ decide_finalize_kernel(const Partial* __restrict__ partials, int splits, int N,
 }  // namespace
 
 int decide_splits(const spiffy_decide_desc& d, int64_t* chunk_elems) {
-  // A slice is what one CTA holds in registers: kReduceThreads * kUnroll vectors
-  // of 16 bytes (8192 bf16 or 4096 fp32 logits); slices start on 16-byte boundaries.
+  // A slice is at most what one CTA holds in registers: kReduceThreads * kUnroll
+  // vectors of 16 bytes (16384 bf16 or 8192 fp32 logits); slices start on
+  // 16-byte boundaries.
   const int64_t epv = d.logits_dtype == SPIFFY_BF16 ? 8 : 4;
-  const int64_t chunk = (int64_t)kReduceThreads * kUnroll * epv;
-  const int64_t splits = (d.vocab + chunk - 1) / chunk;
+  const int64_t most = (int64_t)kReduceThreads * kUnroll * epv;
+  const int64_t splits = (d.vocab + most - 1) / most;
+  // equal slices, rounded up to whole vectors
+  int64_t chunk = (d.vocab + splits - 1) / splits;
+  chunk = (chunk + epv - 1) / epv * epv;
   if (chunk_elems) *chunk_elems = chunk;
   return (int)(splits < 1 ? 1 : splits);
 }
