@@ -39,7 +39,10 @@ sys.path.insert(0, ROOT)
 METRIC = "draft-graph verify steps/sec at LLaDA-8B shape"
 UNIT = "steps/s"
 WORKLOAD = "config2-llada8b: B=1 N=8 L=32 P=512 Hq=Hkv=32 d=128 bf16, V=126464, threshold 0.9"
-N_SETS = 6  # rotating input sets; 6 x 81.5 MB = 489 MB > 126 MB of L2
+N_SETS = 6  # rotating input sets; 6 x 79.4 MB = 477 MB > 126 MB of L2
+# dram__bytes_read.sum + dram__bytes_write.sum of one decide_reduce_kernel launch at this workload
+# (ncu capture summarised under profiles/); set to None whenever that kernel changes
+NCU_REDUCE_TRAFFIC_BYTES = 41.77e6
 
 
 def parse():
@@ -389,7 +392,9 @@ def main():
         "kernel": "decide_reduce_kernel (timed as the spiffy_unmask_decide call: reduce + finalize)",
         "bound": "hbm", "achieved": decide_bytes / t_dec / 1e9, "peak": peaks["hbm_gbs"],
         "unit": "GB/s", "frac": decide_bytes / t_dec / 1e9 / peaks["hbm_gbs"],
-        "peak_source": peaks["source"] + " (burst copy)", "traffic": None,
+        "peak_source": peaks["source"] + " (burst copy)", "traffic": NCU_REDUCE_TRAFFIC_BYTES,
+        "traffic_note": "dram read+write bytes of one decide_reduce_kernel launch, ncu capture in "
+                        "profiles/decide_reduce_kernel_config2.md",
         "algorithmic_bytes": decide_bytes, "seconds": t_dec,
     }
     attn_tc = attn_flops / t_attn / 1e12
