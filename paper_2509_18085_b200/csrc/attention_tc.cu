@@ -53,6 +53,7 @@ constexpr uint32_t kTmemCols = 512;
 // O: 2 x 128 columns, one accumulator per softmax warpgroup
 constexpr uint32_t kColS = 0, kColO = 256;
 constexpr float kRescaleLog2 = 8.0f;
+constexpr int kSoloTiles = 6;  // up to this many key tiles one softmax warpgroup works alone
 
 // NQ M-tiles per CTA: NQ Q tiles, a K ring of 3 stages and a V ring of 4 - NQ
 // stages: 7 tiles of 32 KB either way.
@@ -311,15 +312,22 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int hh = r % p.group;
     const int node = min(nl, p.NL - 1) / p.L;
     const uint32_t lane_base = (uint32_t)(quad * 32);
-    const uint32_t col_s = kColS + (uint32_t)wg * BN;  // this warpgroup's S (and P) buffer
-    const uint32_t col_o = kColO + (uint32_t)wg * HD;  // and its accumulator
+    // With only a few key tiles the hand-over between the warpgroups costs more
+    // than it hides: warpgroup 0 then works alone ("solo") on both buffers, with
+    // one (maximum, sum, tile count) per buffer, and warpgroup 1 sits the CTA out.
+    const bool solo = NQ == 1 && T <= kSoloTiles;
     const float k2 = p.scale_log2;
-    float m_run = -INFINITY, l_run = 0.f;
+    float m_run = -INFINITY, l_run = 0.f;  // state of the buffer in hand
+    float m_alt = -INFINITY, l_alt = 0.f;  // solo: state of the other buffer
     bool ok = true;
-    int mine = 0;  // tiles this warpgroup has finished
-    for (int j = (NQ == 1 ? wg : 0); j < T; j += (NQ == 1 ? 2 : 1), ++mine) {
+    int mine = 0, mine_alt = 0;  // tiles finished on the buffer in hand / on the other one
+    const int j_step = (NQ == 1 && !solo) ? 2 : 1;
+    for (int j = (NQ == 1 && !solo) ? wg : 0; j < T && !(solo && wg == 1); j += j_step) {
+      const int bi = solo ? (j & 1) : wg;                // S/P buffer and accumulator of this tile
+      const uint32_t col_s = kColS + (uint32_t)bi * BN;
+      const uint32_t col_o = kColO + (uint32_t)bi * HD;
       // wait outcomes are made warp-uniform: the TMEM accesses below are warp-collective
-      if (!__all_sync(0xffffffffu, mbar_wait(s_full + wg, (uint32_t)mine & 1u, abort_flag))) {
+      if (!__all_sync(0xffffffffu, mbar_wait(s_full + bi, (uint32_t)mine & 1u, abort_flag))) {
         ok = false;
         break;
       }
@@ -361,7 +369,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         }
         if (mine > 0) {  // the accumulator holds this warpgroup's earlier tiles: wait, then rescale
           if (!__all_sync(0xffffffffu,
-                          mbar_wait(pv_done + wg, (uint32_t)(mine - 1) & 1u, abort_flag))) {
+                          mbar_wait(pv_done + bi, (uint32_t)(mine - 1) & 1u, abort_flag))) {
             ok = false;
             break;
           }
@@ -395,15 +403,29 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
       tmem_st_x64(tmem_addr(tmem, lane_base, col_s), pk);
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(p_ready + wg);
+      mbar_arrive(p_ready + bi);
+      ++mine;
+      if (solo) {  // the other buffer is next
+        float t = m_run; m_run = m_alt; m_alt = t;
+        t = l_run; l_run = l_alt; l_alt = t;
+        const int c = mine; mine = mine_alt; mine_alt = c;
+      }
     }
+    // solo: "in hand" is now buffer T & 1; name the two by buffer instead
+    const int buf_hand = solo ? (T & 1) : wg;
+    const uint32_t col_s = kColS + (uint32_t)buf_hand * BN;
+    const uint32_t col_o = kColO + (uint32_t)buf_hand * HD;
     // ------------------------------------------------------------ epilogue --
     // Each warpgroup waits for its own accumulator, the two exchange their
     // (reference maximum, sum) per row through two spare tensor-memory columns
     // of their S buffers, and each then merges and stores one half of the
     // columns of every row.
     if (ok && mine > 0)
-      ok = __all_sync(0xffffffffu, mbar_wait(pv_done + wg, (uint32_t)(mine - 1) & 1u, abort_flag));
+      ok = __all_sync(0xffffffffu,
+                      mbar_wait(pv_done + buf_hand, (uint32_t)(mine - 1) & 1u, abort_flag));
+    if (ok && solo && mine_alt > 0)
+      ok = __all_sync(0xffffffffu, mbar_wait(pv_done + (buf_hand ^ 1), (uint32_t)(mine_alt - 1) & 1u,
+                                             abort_flag));
     if constexpr (NQ == 2) {
       // each warpgroup owns its rows outright: normalise (or hand on the partial) and store
       if (ok) {
@@ -441,19 +463,23 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
           pml[1] = l_run;
         }
       }
-    } else {
-    constexpr uint32_t kColMl = BN / 2;  // first S column that no P lies over
-    tmem_st_x2(tmem_addr(tmem, lane_base, col_s + kColMl), __float_as_uint(m_run),
-               __float_as_uint(l_run));
-    tmem_wait_st();
-    tc_fence_before_sync();
-    asm volatile("bar.sync 1, 256;" ::: "memory");  // all eight softmax warps, whatever `ok` says
-    tc_fence_after_sync();
-    uint32_t um, ul;
-    tmem_ld_x2(tmem_addr(tmem, lane_base, kColS + (uint32_t)(wg ^ 1) * BN + kColMl), um, ul);
-    const float m_o = __uint_as_float(um), l_o = __uint_as_float(ul);  // the other warpgroup's
-    const float m_a = wg == 0 ? m_run : m_o, l_a = wg == 0 ? l_run : l_o;
-    const float m_b = wg == 0 ? m_o : m_run, l_b = wg == 0 ? l_o : l_run;
+    } else if (!(solo && wg == 1)) {
+    float m_o = m_alt, l_o = l_alt;  // state of the other buffer
+    if (!solo) {
+      constexpr uint32_t kColMl = BN / 2;  // first S column that no P lies over
+      tmem_st_x2(tmem_addr(tmem, lane_base, col_s + kColMl), __float_as_uint(m_run),
+                 __float_as_uint(l_run));
+      tmem_wait_st();
+      tc_fence_before_sync();
+      asm volatile("bar.sync 1, 256;" ::: "memory");  // all eight softmax warps, whatever `ok` says
+      tc_fence_after_sync();
+      uint32_t um, ul;
+      tmem_ld_x2(tmem_addr(tmem, lane_base, kColS + (uint32_t)(wg ^ 1) * BN + kColMl), um, ul);
+      m_o = __uint_as_float(um);
+      l_o = __uint_as_float(ul);
+    }
+    const float m_a = buf_hand == 0 ? m_run : m_o, l_a = buf_hand == 0 ? l_run : l_o;
+    const float m_b = buf_hand == 0 ? m_o : m_run, l_b = buf_hand == 0 ? l_o : l_run;
     const float m_all = fmaxf(m_a, m_b);
     // an accumulator whose warpgroup saw no key of this row (or no tile at all) is left out
     const bool has_a = m_a != -INFINITY, has_b = m_b != -INFINITY;
@@ -468,7 +494,8 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
           p.out + (((int64_t)b * p.NL + nl) * p.Hq + (int64_t)g * p.group + hh) * HD;
       float* po = p.part_o + (tile * BM + r) * HD;
 #pragma unroll
-      for (int c0 = wg * 64; c0 < wg * 64 + 64; c0 += 32) {
+      // solo: all 128 columns; otherwise each warpgroup stores one half
+      for (int c0 = solo ? 0 : wg * 64; c0 < (solo ? HD : wg * 64 + 64); c0 += 32) {
         uint32_t oa[32], ob[32];
         tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + c0), oa);
         tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + HD + c0), ob);
