@@ -19,7 +19,10 @@
 namespace spiffy {
 namespace {
 
-constexpr int kReduceThreads = 256;
+#ifndef SPIFFY_DECIDE_THREADS
+#define SPIFFY_DECIDE_THREADS 128
+#endif
+constexpr int kReduceThreads = SPIFFY_DECIDE_THREADS;
 #ifndef SPIFFY_DECIDE_UNROLL
 #define SPIFFY_DECIDE_UNROLL 8
 #endif
@@ -163,7 +166,7 @@ decide_reduce_kernel(const T* __restrict__ logits, int64_t row_stride, int V,
   const uint4* p = reinterpret_cast<const uint4*>(base + begin);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-  // 1. the thread's vectors t, t + 256, ...; thread 0 also takes the ragged tail
+  // 1. the thread's vectors t, t + kReduceThreads, ...; thread 0 also takes the ragged tail
   uint4 v[kUnroll];
 #pragma unroll
   for (int u = 0; u < kUnroll; ++u)
@@ -316,7 +319,7 @@ decide_finalize_kernel(const Partial* __restrict__ partials, int splits, int N,
 
 int decide_splits(const spiffy_decide_desc& d, int64_t* chunk_elems) {
   // A slice is at most what one CTA holds in registers: kReduceThreads * kUnroll
-  // vectors of 16 bytes (16384 bf16 or 8192 fp32 logits); slices start on
+  // vectors of 16 bytes (8192 bf16 or 4096 fp32 logits); slices start on
   // 16-byte boundaries.
   const int64_t epv = d.logits_dtype == SPIFFY_BF16 ? 8 : 4;
   const int64_t most = (int64_t)kReduceThreads * kUnroll * epv;
