@@ -36,7 +36,8 @@ def oracle_attention(w, scale=None):
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
-@pytest.mark.parametrize("index,n_nodes", [(1, None), (2, None), (3, None), (5, 1), (5, 8), (5, 64)])
+@pytest.mark.parametrize("index,n_nodes", [(1, None), (2, None), (3, None), (5, 1), (5, 2), (5, 4), (5, 8),
+                                           (5, 16), (5, 32), (5, 64)])
 def test_configs(index, n_nodes, kernel):
     cfg = W.config(index, n_nodes)
     w = W.make(cfg, W.seed_for(index, 0), decision=False)

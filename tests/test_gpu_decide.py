@@ -15,7 +15,8 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("index,n_nodes,cases", [(1, None, 10), (2, None, 2), (3, None, 2),
-                                                 (5, 1, 2), (5, 8, 1), (5, 64, 1)])
+                                                 (5, 1, 2), (5, 2, 1), (5, 4, 1), (5, 8, 1), (5, 16, 1),
+                                                 (5, 32, 1), (5, 64, 1)])
 def test_configs_sharp(index, n_nodes, cases):
     hops = []
     for case in range(cases):

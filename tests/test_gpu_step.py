@@ -91,3 +91,37 @@ def test_losslessness_with_the_cuda_library(rule, S, tau, seed):
         assert model.calls == calls - sum(accepted)
         total += sum(accepted)
     assert total > 0
+
+
+def test_graph_replay_at_the_benchmark_configuration_matches_the_oracle():
+    """The launch configuration the benchmark times: one verification step of
+    the LLaDA-8B-shaped configuration captured in a CUDA graph and replayed.
+    Decisions and the walk are compared bit-exactly, confidences and a sample of
+    attention rows within tolerance."""
+    from paper_2509_18085_b200.step import VerifyStep, inputs_from_workload
+    cfg = W.config(2)
+    w = W.make(cfg, W.seed_for(2, 100))
+    x = inputs_from_workload(w)
+    step = VerifyStep(cfg)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        step.run(x)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            step.run(x)
+        step.attn_out.zero_()
+        step.decision.top_tok.zero_()
+        step.walk.next_block.zero_()
+        for _ in range(3):
+            graph.replay()
+        stream.synchronize()
+    odec, owalk = G.oracle_decide(w)
+    n = G.assert_decision_parity(w, step.decision, step.walk, odec, owalk, G.TOL["bf16"], G.MARGIN["bf16"])
+    assert n == cfg.batch
+    got = step.attn_out.float().cpu().numpy()
+    for node in (0, 3, 7):
+        want = oracle.graph_attention(w.q[:, node:node + 1], w.k_prefix, w.v_prefix,
+                                      w.k_block[:, node:node + 1], w.v_block[:, node:node + 1])
+        assert np.max(np.abs(got[:, node] - want[:, 0])) <= G.TOL["bf16"]
+    assert int(step.attn_status.item()) == 0
