@@ -248,6 +248,65 @@ spiffy_status spiffy_accept_walk(const spiffy_decide_desc* desc,
                                  int32_t* path, int32_t* next_block,
                                  int32_t* dev_status, void* cuda_stream);
 
+/* ------------------------------------------------------------------------- */
+/* Drafting and pruning (Sec. 4.4.2 "Drafting Source", Sec. 4.4.4 "Pruning")  */
+/* ------------------------------------------------------------------------- */
+typedef struct {
+  int32_t batch;         /* B                                                */
+  int32_t block_len;     /* L in [1, 64]                                     */
+  int32_t vocab;         /* V                                                */
+  int32_t logits_dtype;  /* spiffy_dtype                                     */
+  int64_t row_stride;    /* elements between logits rows, as in the decision */
+  int32_t mask_token_id;
+  int32_t n_formulas;    /* D draft formulas of the calibrated graph, <= 1024 */
+  int32_t top_k;         /* vocabulary ranks a formula may use, 1..4         */
+  int32_t budget;        /* D* drafts kept after pruning, 1..D               */
+  int32_t parent_cap;    /* entries per sequence in parent_idx               */
+} spiffy_draft_desc;
+
+size_t spiffy_draft_blocks_workspace(const spiffy_draft_desc* desc);
+
+/*
+ * Builds the draft blocks of the next verification step from the target
+ * distribution of the current block.  Per sequence: the still-masked positions
+ * are ranked by their maximum probability (token position rank i, 0 = most
+ * confident; ties to the lower position) and per position the vocabulary by
+ * probability (vocabulary rank j; ties to the lower token id); candidate c_ij
+ * is the token of rank j at the position of rank i (Sec. 4.4.2).  Draft formula
+ * q is a fixed list of (i, j) pairs from the offline calibration; its block is
+ * the current block with its candidates written in.  Pruning (Sec. 4.4.4):
+ * localScore = geometric mean of the candidates' probabilities, childScore =
+ * geometric mean of the local scores of the formula's children, score = their
+ * geometric mean (just localScore without children); the `budget` best formulas
+ * are kept (ties to the lower index).  A formula that asks for a position rank
+ * beyond the number of masked positions cannot be built: score -inf, never kept.
+ *
+ *   logits      [B][L] rows of V: the distribution to draft from (that of the
+ *               node accepted last); rows of unmasked positions are not read
+ *   state       [B][L] int32 current block
+ *   formula_off [D+1], formula_i, formula_j: CSR of the (i, j) pairs, shared
+ *               by all sequences; parents before children
+ *   child_off   [D+1], child_idx: children of each formula in the draft graph
+ *   draft_tokens [B][D*+1][L]: node 0 = the current block, then the kept drafts
+ *               in formula order; unused nodes repeat the current block
+ *   kept        [B][D*] formula index of every kept draft, -1 for unused nodes
+ *   score       [B][D] fp32 score of every formula
+ *   parent_off  [B][D*+2], parent_idx [B][parent_cap]: parent lists over the
+ *               D*+1 nodes in the layout spiffy_accept_walk reads: node a is a
+ *               parent of node c when a's candidate set is a strict subset of
+ *               c's (Eqs. draft-graph-2/3; node 0 is the empty set)
+ *   dev_status  [B]: SPIFFY_DEV_NONFINITE for an unusable logits row,
+ *               SPIFFY_DEV_BADGRAPH when parent_cap was too small (lists cut)
+ */
+spiffy_status spiffy_draft_blocks(const spiffy_draft_desc* desc, const void* logits,
+                                  const int32_t* state, const int32_t* formula_off,
+                                  const int32_t* formula_i, const int32_t* formula_j,
+                                  const int32_t* child_off, const int32_t* child_idx,
+                                  int32_t* draft_tokens, int32_t* kept, float* score,
+                                  int32_t* parent_off, int32_t* parent_idx,
+                                  int32_t* dev_status, void* workspace,
+                                  size_t workspace_bytes, void* cuda_stream);
+
 /* Static description of a status code; never NULL. */
 const char* spiffy_status_string(spiffy_status status);
 

@@ -51,6 +51,18 @@ spiffy_status check_decide_desc(const spiffy_decide_desc* d, bool need_vocab) {
   return SPIFFY_OK;
 }
 
+spiffy_status check_draft_desc(const spiffy_draft_desc* d) {
+  if (!d) return SPIFFY_EINVAL;
+  if (d->batch < 1 || d->block_len < 1 || d->vocab < 1 || d->n_formulas < 1) return SPIFFY_EINVAL;
+  if (d->logits_dtype != SPIFFY_F32 && d->logits_dtype != SPIFFY_BF16) return SPIFFY_EINVAL;
+  if (d->row_stride < d->vocab) return SPIFFY_EINVAL;
+  if ((d->row_stride * (d->logits_dtype == SPIFFY_BF16 ? 2 : 4)) % 16 != 0) return SPIFFY_EINVAL;
+  if (d->top_k < 1 || d->budget < 1 || d->budget > d->n_formulas || d->parent_cap < 1) return SPIFFY_EINVAL;
+  if (d->block_len > 64 || d->top_k > 4 || d->n_formulas > 1024) return SPIFFY_EUNSUPPORTED;
+  if ((int64_t)d->batch * d->block_len > 65535) return SPIFFY_EUNSUPPORTED;
+  return SPIFFY_OK;
+}
+
 }  // namespace
 }  // namespace spiffy
 
@@ -131,6 +143,32 @@ spiffy_status spiffy_accept_walk(const spiffy_decide_desc* desc,
   return launch_walk(*desc, block_tokens, parent_off, parent_idx, parent_cap,
                      top_tok, unmask_bits, accepted_node, n_accepted, path,
                      next_block, dev_status, static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t spiffy_draft_blocks_workspace(const spiffy_draft_desc* desc) {
+  if (check_draft_desc(desc) != SPIFFY_OK) return 0;
+  return draft_workspace_bytes(*desc);
+}
+
+spiffy_status spiffy_draft_blocks(const spiffy_draft_desc* desc, const void* logits,
+                                  const int32_t* state, const int32_t* formula_off,
+                                  const int32_t* formula_i, const int32_t* formula_j,
+                                  const int32_t* child_off, const int32_t* child_idx,
+                                  int32_t* draft_tokens, int32_t* kept, float* score,
+                                  int32_t* parent_off, int32_t* parent_idx,
+                                  int32_t* dev_status, void* workspace,
+                                  size_t workspace_bytes, void* cuda_stream) {
+  const spiffy_status st = check_draft_desc(desc);
+  if (st != SPIFFY_OK) return st;
+  if (!logits || !state || !formula_off || !formula_i || !formula_j || !child_off || !child_idx ||
+      !draft_tokens || !kept || !score || !parent_off || !parent_idx)
+    return SPIFFY_EINVAL;
+  if (!aligned16(logits)) return SPIFFY_EINVAL;
+  const size_t need = draft_workspace_bytes(*desc);
+  if (!workspace || workspace_bytes < need || !aligned16(workspace)) return SPIFFY_EWORKSPACE;
+  return launch_draft(*desc, logits, state, formula_off, formula_i, formula_j, child_off, child_idx,
+                      draft_tokens, kept, score, parent_off, parent_idx, dev_status, workspace,
+                      static_cast<cudaStream_t>(cuda_stream));
 }
 
 const char* spiffy_status_string(spiffy_status status) {

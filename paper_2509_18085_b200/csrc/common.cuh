@@ -37,6 +37,14 @@ spiffy_status launch_attention_simt(const spiffy_attn_desc& d, const void* q,
                                     const void* kb, const void* vb, void* out,
                                     cudaStream_t stream);
 
+size_t draft_workspace_bytes(const spiffy_draft_desc& d);
+spiffy_status launch_draft(const spiffy_draft_desc& d, const void* logits, const int32_t* state,
+                           const int32_t* formula_off, const int32_t* formula_i,
+                           const int32_t* formula_j, const int32_t* child_off,
+                           const int32_t* child_idx, int32_t* tokens, int32_t* kept, float* score,
+                           int32_t* parent_off, int32_t* parent_idx, int32_t* dev_status, void* ws,
+                           cudaStream_t stream);
+
 // tcgen05 path: shape support query, workspace and launch.
 bool attention_tc_supported(const spiffy_attn_desc& d);
 size_t attention_tc_workspace_bytes(const spiffy_attn_desc& d);

@@ -27,7 +27,7 @@ EXPORTS = (
     "spiffy_graph_attention_workspace", "spiffy_graph_attention",
     "spiffy_unmask_decide_workspace", "spiffy_unmask_decide",
     "spiffy_accept_walk", "spiffy_status_string", "spiffy_launch_count",
-    "spiffy_unmask_decide_static",
+    "spiffy_unmask_decide_static", "spiffy_draft_blocks_workspace", "spiffy_draft_blocks",
 )
 DECIDE_STATIC_BYTES = 2 << 20
 
@@ -55,6 +55,13 @@ class DecideDesc(ctypes.Structure):
                 ("top_s", ctypes.c_int32), ("threshold", ctypes.c_float)]
 
 
+class DraftDesc(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("block_len", ctypes.c_int32), ("vocab", ctypes.c_int32),
+                ("logits_dtype", ctypes.c_int32), ("row_stride", ctypes.c_int64),
+                ("mask_token_id", ctypes.c_int32), ("n_formulas", ctypes.c_int32),
+                ("top_k", ctypes.c_int32), ("budget", ctypes.c_int32), ("parent_cap", ctypes.c_int32)]
+
+
 _lib = None
 
 
@@ -78,6 +85,10 @@ def lib() -> ctypes.CDLL:
         L.spiffy_unmask_decide.argtypes = [ctypes.POINTER(DecideDesc)] + [vp] * 8 + [sz, vp]
         L.spiffy_unmask_decide_static.restype = ctypes.c_int
         L.spiffy_unmask_decide_static.argtypes = [ctypes.POINTER(DecideDesc)] + [vp] * 8
+        L.spiffy_draft_blocks_workspace.restype = sz
+        L.spiffy_draft_blocks_workspace.argtypes = [ctypes.POINTER(DraftDesc)]
+        L.spiffy_draft_blocks.restype = ctypes.c_int
+        L.spiffy_draft_blocks.argtypes = [ctypes.POINTER(DraftDesc)] + [vp] * 14 + [sz, vp]
         L.spiffy_accept_walk.restype = ctypes.c_int
         L.spiffy_accept_walk.argtypes = [ctypes.POINTER(DecideDesc), vp, vp, vp, i32] + [vp] * 8
         L.spiffy_status_string.restype = ctypes.c_char_p
@@ -269,4 +280,82 @@ def spiffy_accept_walk(block_tokens, parent_off, parent_idx, top_tok, unmask_bit
         _dev(out.next_block, "next_block", torch.int32),
         _dev(out.dev_status, "dev_status", torch.int32), _stream(stream))
     _check(st, "spiffy_accept_walk")
+    return out
+
+
+@dataclass
+class DraftGraph:
+    """The calibrated draft graph on the device: D formulas of (position rank,
+    vocabulary rank) pairs and each formula's children, both in CSR form."""
+    formula_off: torch.Tensor  # [D+1] int32
+    formula_i: torch.Tensor
+    formula_j: torch.Tensor
+    child_off: torch.Tensor    # [D+1] int32
+    child_idx: torch.Tensor
+
+    @property
+    def n_formulas(self) -> int:
+        return self.formula_off.numel() - 1
+
+
+def draft_graph(formulas, children, device="cuda") -> DraftGraph:
+    """formulas: list of lists of (i, j); children: list of lists of formula indices."""
+    def csr(lists, width):
+        off, flat = [0], []
+        for x in lists:
+            flat += list(x)
+            off.append(len(flat))
+        flat = flat or [(0,) * width if width > 1 else 0]
+        return off, flat
+    foff, pairs = csr(formulas, 2)
+    coff, kids = csr(children, 1)
+    t = lambda a: torch.tensor(a, dtype=torch.int32, device=device)
+    return DraftGraph(t(foff), t([p[0] for p in pairs]), t([p[1] for p in pairs]), t(coff), t(kids))
+
+
+@dataclass
+class Drafts:
+    tokens: torch.Tensor      # [B, D*+1, L] int32
+    kept: torch.Tensor        # [B, D*] int32
+    score: torch.Tensor       # [B, D] float32
+    parent_off: torch.Tensor  # [B, D*+2] int32
+    parent_idx: torch.Tensor  # [B, cap] int32
+    dev_status: torch.Tensor  # [B] int32
+
+
+def spiffy_draft_blocks(logits, state, mask_token_id: int, graph: DraftGraph, budget: int, top_k: int,
+                        parent_cap: int = 0, out: Optional[Drafts] = None, workspace=None,
+                        stream=None) -> Drafts:
+    """Drafting and pruning.  logits [B,L,V] (rows may be a strided view), state [B,L] int32."""
+    B, L = state.shape
+    V = logits.shape[-1]
+    D = graph.n_formulas
+    cap = parent_cap or max(4, (budget + 1) * budget // 2)
+    row_stride = logits.stride(-2)
+    if B > 1 and logits.stride(0) != L * row_stride:
+        raise ValueError("logits rows must be equally spaced")
+    desc = DraftDesc(B, L, V, _dtype_code(logits), int(row_stride), int(mask_token_id), D, int(top_k),
+                     int(budget), int(cap))
+    dev = logits.device
+    if out is None:
+        out = Drafts(torch.empty((B, budget + 1, L), dtype=torch.int32, device=dev),
+                     torch.empty((B, budget), dtype=torch.int32, device=dev),
+                     torch.empty((B, D), dtype=torch.float32, device=dev),
+                     torch.empty((B, budget + 2), dtype=torch.int32, device=dev),
+                     torch.zeros((B, cap), dtype=torch.int32, device=dev),
+                     torch.zeros((B,), dtype=torch.int32, device=dev))
+    need = int(lib().spiffy_draft_blocks_workspace(ctypes.byref(desc)))
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    i32 = torch.int32
+    st = lib().spiffy_draft_blocks(
+        ctypes.byref(desc), _logits_ptr(logits) if logits.dim() == 4 else logits.data_ptr(),
+        _dev(state, "state", i32), _dev(graph.formula_off, "formula_off", i32),
+        _dev(graph.formula_i, "formula_i", i32), _dev(graph.formula_j, "formula_j", i32),
+        _dev(graph.child_off, "child_off", i32), _dev(graph.child_idx, "child_idx", i32),
+        _dev(out.tokens, "tokens", i32), _dev(out.kept, "kept", i32),
+        _dev(out.score, "score", torch.float32), _dev(out.parent_off, "parent_off", i32),
+        _dev(out.parent_idx, "parent_idx", i32), _dev(out.dev_status, "dev_status", i32),
+        _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(st, "spiffy_draft_blocks")
     return out
