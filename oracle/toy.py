@@ -242,3 +242,25 @@ def random_drafter(mask_id, n_drafts=4, seed=0, vocab=None):
         return np.asarray(out, dtype=np.int32).reshape(-1, len(state))
 
     return drafter
+
+
+def auto_drafter(model, formulas, children, budget, top_k, draft=None):
+    """Auto-speculation (Sec. 4.4.2): drafts are built from the target
+    distribution of the current block with fixed draft formulas and pruned to
+    ``budget`` (Sec. 4.4.4).  ``model`` is a twin of the decoder's model (same
+    weights), so that the decoder's own call count is not disturbed; ``draft``
+    replaces the oracle's drafting step (the CUDA library in the GPU tests)."""
+    from . import drafting
+
+    def default_draft(logits, state, mask_id):
+        return drafting.draft_blocks(logits, state, mask_id, formulas, children, budget, top_k).tokens
+
+    build = draft or default_draft
+
+    def drafter(state, call):
+        logits = model(state[None])[:, 0]  # [1, L, V]: p_TD of the current block
+        tokens = build(np.ascontiguousarray(logits, dtype=np.float32), state[None].astype(np.int32),
+                       model.mask_id)
+        return np.asarray(tokens)[0, 1:]
+
+    return drafter

@@ -125,3 +125,32 @@ def test_graph_replay_at_the_benchmark_configuration_matches_the_oracle():
                                       w.k_block[:, node:node + 1], w.v_block[:, node:node + 1])
         assert np.max(np.abs(got[:, node] - want[:, 0])) <= G.TOL["bf16"]
     assert int(step.attn_status.item()) == 0
+
+
+def test_auto_speculation_through_the_cuda_drafting_call():
+    """The closed loop of the method on the toy model: draft with
+    spiffy_draft_blocks, verify with the CUDA decision and walk; the trajectory
+    is plain decoding's and accepted drafts save model calls."""
+    formulas = [[(0, 0)], [(0, 1)], [(0, 0), (1, 0)], [(0, 0), (1, 1)], [(0, 0), (1, 0), (2, 0)]]
+    children = [[2, 3], [], [4], [], []]
+    graph = spiffy.draft_graph(formulas, children)
+    _, decide, walk = gpu_backends()
+
+    def draft(logits, state, mask_id):
+        d = spiffy.spiffy_draft_blocks(G.to_dev(logits), G.to_dev(state), mask_id, graph, 3, 2)
+        return d.tokens.cpu().numpy()
+
+    saved = 0
+    for seed in range(3):
+        start = np.full(8, 23, dtype=np.int32)
+        start[seed] = seed + 1
+        model = toy.ToyModel(seed=seed)
+        vanilla = toy.vanilla_decode(model, start, oracle.RULE_TOPS, decide=decide)
+        calls = model.calls
+        model.calls = 0
+        drafter = toy.auto_drafter(toy.ToyModel(seed=seed), formulas, children, 3, 2, draft=draft)
+        traj, accepted = toy.speculative_decode(model, start, drafter, oracle.RULE_TOPS, decide=decide, walk=walk)
+        assert len(traj) == len(vanilla) and all(np.array_equal(a, b) for a, b in zip(traj, vanilla))
+        assert model.calls == calls - sum(accepted)
+        saved += sum(accepted)
+    assert saved > 0

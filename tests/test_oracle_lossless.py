@@ -72,3 +72,24 @@ def test_a_planted_mistake_breaks_the_invariant():
             np.array_equal(a, b) for a, b in zip(traj, vanilla_bad))
         diverged += not same
     assert diverged > 0
+
+
+def test_auto_speculation_with_the_drafting_oracle_is_lossless_and_saves_calls():
+    """Drafts built from the target distribution with fixed formulas (Sec. 4.4.2)
+    and pruned (Sec. 4.4.4): the first-rank chain is what plain decoding does
+    next, so drafts are accepted, and the trajectory stays the plain one."""
+    formulas = [[(0, 0)], [(0, 1)], [(0, 0), (1, 0)], [(0, 0), (1, 1)], [(0, 0), (1, 0), (2, 0)]]
+    children = [[2, 3], [], [4], [], []]
+    saved = 0
+    for seed in range(4):
+        model = toy.ToyModel(seed=seed)
+        s0 = start_state(model, seed)
+        vanilla = toy.vanilla_decode(model, s0, oracle.RULE_TOPS)
+        calls_vanilla = model.calls
+        model.calls = 0
+        drafter = toy.auto_drafter(toy.ToyModel(seed=seed), formulas, children, budget=3, top_k=2)
+        traj, accepted = toy.speculative_decode(model, s0, drafter, oracle.RULE_TOPS)
+        assert len(traj) == len(vanilla) and all(np.array_equal(a, b) for a, b in zip(traj, vanilla))
+        assert model.calls == calls_vanilla - sum(accepted)
+        saved += sum(accepted)
+    assert saved > 0
