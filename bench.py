@@ -55,7 +55,7 @@ def parse():
     ap.add_argument("--nodes", type=int, default=None, help="node count for configuration 5")
     ap.add_argument("--attn-kernel", default="auto", choices=["auto", "simt", "tcgen05"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--part", default="step", choices=["step", "attention", "decide"],
+    ap.add_argument("--part", default="step", choices=["step", "attention", "decide", "draft"],
                     help="time one library call alone on any configuration (for profiling); "
                          "the benchmark line itself is --part step")
     ap.add_argument("--sets", type=int, default=0, help="rotating input sets for --part (0 = enough to exceed L2)")
@@ -230,6 +230,8 @@ def run_part(args):
 
     torch.cuda.set_device(0)
     cfg = W.config(args.config, args.nodes)
+    if args.part == "draft":
+        return run_draft_part(args, cfg)
     attn = args.part == "attention"
     probe = W.make(cfg, W.seed_for(args.config, 100), attention=attn, decision=not attn)
     masked = int((probe.block_tokens == cfg.mask_id).sum())
@@ -276,6 +278,55 @@ def run_part(args):
                    masked_rows=masked_all)
     out["peaks"] = peaks["source"]
     print(json.dumps(out))
+
+
+def run_draft_part(args, cfg):
+    """spiffy_draft_blocks alone (drafting + pruning from the true block's
+    distribution): ten formulas over position ranks 0..3 and vocabulary ranks
+    0..2, pruned to three drafts -- the paper's operating point (D = 10, D* = 3)."""
+    import torch
+    from paper_2509_18085_b200 import spiffy
+    from paper_2509_18085_b200 import workloads as W
+    formulas = [[(0, 0)], [(0, 1)], [(1, 0)], [(0, 0), (1, 0)], [(0, 0), (1, 1)], [(0, 1), (1, 0)],
+                [(0, 0), (2, 0)], [(0, 0), (1, 0), (2, 0)], [(0, 0), (1, 0), (2, 2)],
+                [(0, 0), (1, 0), (2, 0), (3, 0)]]
+    children = [[3, 4, 6], [5], [3, 5], [7, 8], [], [], [7], [9], [], []]
+    graph = spiffy.draft_graph(formulas, children)
+    n_sets = args.sets or 24
+    dt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    sets, masked = [], 0
+    for i in range(n_sets):
+        w = W.make(W.config(args.config, 1), W.seed_for(args.config, 300 + i), attention=False)
+        sets.append((torch.from_numpy(w.logits[:, 0]).to(dt).cuda(), torch.from_numpy(w.block_tokens[:, 0]).cuda()))
+        masked += int((w.block_tokens[:, 0] == cfg.mask_id).sum())
+    out = spiffy.spiffy_draft_blocks(sets[0][0], sets[0][1], cfg.mask_id, graph, 3, 3)
+    ws = torch.empty(1 << 22, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        call = lambda x: spiffy.spiffy_draft_blocks(x[0], x[1], cfg.mask_id, graph, 3, 3, out=out, workspace=ws)
+        for x in sets:
+            call(x)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for x in sets:
+                call(x)
+        g.replay()
+        stream.synchronize()
+        reps = max(1, args.steps // n_sets)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        e1.record(stream)
+        stream.synchronize()
+        sec = e0.elapsed_time(e1) * 1e-3 / (reps * n_sets)
+    by = masked / n_sets * cfg.vocab * (2 if cfg.dtype == "bf16" else 4)
+    peaks = measured_peaks()
+    print(json.dumps({"part": "draft", "config": f"config{args.config}-{cfg.name}", "us_per_call": sec * 1e6,
+                      "formulas": len(formulas), "budget": 3, "top_k": 3, "masked_rows": masked / n_sets,
+                      "algorithmic_bytes": by, "gbs": by / sec / 1e9, "frac_of_hbm": by / sec / 1e9 / peaks["hbm_gbs"],
+                      "input_sets": n_sets, "peaks": peaks["source"], "dev_status": int(out.dev_status.max())}))
 
 
 def main():

@@ -22,7 +22,7 @@ namespace {
 constexpr int kThreads = 128;  // top-k kernel
 constexpr int kVecs = 8;       // 128-bit vectors per thread
 constexpr int kMaxK = 4;       // vocabulary ranks
-constexpr int kBuildThreads = 256;
+constexpr int kBuildThreads = 1024;  // a warp per block position
 
 struct __align__(16) TopPartial {
   float m, s;          // slice maximum, sum of exp(x - m)
@@ -206,7 +206,7 @@ __device__ bool strict_subset(const BuildArgs& g, int a, int c) {
   return true;
 }
 
-// grid = B sequences, 256 threads; dynamic shared memory, see the carve-up below.
+// grid = B sequences, 1024 threads; dynamic shared memory, see the carve-up below.
 __global__ void __launch_bounds__(kBuildThreads)
 draft_build_kernel(const BuildArgs g) {
 #if __CUDA_ARCH__ >= 900
@@ -252,25 +252,39 @@ draft_build_kernel(const BuildArgs g) {
     }
     if (lane == 0 && (!(fabsf(m) < INFINITY) || !(s >= 1.0f) || !(s < INFINITY)) && g.dev_status)
       atomicOr(g.dev_status + b, SPIFFY_DEV_NONFINITE);
-    // K rounds over the splits * K slice candidates (value desc, id asc); a taken one is remembered by its id
-    int taken[kMaxK];
+    // the K best of the splits * K slice candidates (value desc, id asc): every lane
+    // first sorts the candidates it reads (each is read once), then K rounds pick the
+    // best head over the lanes and pop it
+    float hv[kMaxK];
+    int hi[kMaxK];
+#pragma unroll
+    for (int t = 0; t < kMaxK; ++t) { hv[t] = -INFINITY; hi[t] = 0x7fffffff; }
+    for (int c = lane; c < g.splits * K; c += 32) {
+      float v = p[c / K].val[c % K];
+      int i = p[c / K].idx[c % K];
+      if (v == -INFINITY) continue;
+#pragma unroll
+      for (int t = 0; t < kMaxK; ++t)  // insertion into the sorted list
+        if (ahead(v, i, hv[t], hi[t])) {
+          const float tv = hv[t]; const int ti = hi[t];
+          hv[t] = v; hi[t] = i; v = tv; i = ti;
+        }
+    }
     for (int r = 0; r < K; ++r) {
-      float bv = -INFINITY;
-      int bi = 0x7fffffff;
-      for (int c = lane; c < g.splits * K; c += 32) {
-        const float v = p[c / K].val[c % K];
-        const int i = p[c / K].idx[c % K];
-        bool used = false;
-        for (int t = 0; t < r; ++t) used |= taken[t] == i;
-        if (!used && v != -INFINITY && ahead(v, i, bv, bi)) { bv = v; bi = i; }
-      }
+      float bv = hv[0];
+      int bi = hi[0];
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) {
         const float v2 = __shfl_xor_sync(0xffffffffu, bv, off);
         const int i2 = __shfl_xor_sync(0xffffffffu, bi, off);
         if (ahead(v2, i2, bv, bi)) { bv = v2; bi = i2; }
       }
-      taken[r] = bi;
+      if (hi[0] == bi && bv != -INFINITY) {  // this lane's head won: pop it
+#pragma unroll
+        for (int t = 0; t + 1 < kMaxK; ++t) { hv[t] = hv[t + 1]; hi[t] = hi[t + 1]; }
+        hv[kMaxK - 1] = -INFINITY;
+        hi[kMaxK - 1] = 0x7fffffff;
+      }
       if (lane == 0) {
         cand_tok[l * kMaxK + r] = bi;
         cand_p[l * kMaxK + r] = bv == -INFINITY ? 0.f : ex2((bv - m) * kLog2e) / s;

@@ -97,6 +97,32 @@ def test_walk_rejects_bad_arguments(lib):
     assert lib.spiffy_accept_walk(ctypes.byref(d), *neg) == spiffy.EINVAL
 
 
+def test_draft_rejects_bad_arguments(lib):
+    fake = ctypes.c_void_p(0x1000)
+
+    def desc(**kw):
+        d = spiffy.DraftDesc(1, 8, 1024, spiffy.BF16, 1024, 1023, 10, 3, 3, 16)
+        for k, v in kw.items():
+            setattr(d, k, v)
+        return d
+
+    def call(d, ws=fake, ws_bytes=1 << 30, logits=fake):
+        return lib.spiffy_draft_blocks(ctypes.byref(d), logits, *([fake] * 11), None, ws, ws_bytes, None)
+
+    assert lib.spiffy_draft_blocks_workspace(ctypes.byref(desc())) > 0
+    assert call(desc(), ws=None) == spiffy.EWORKSPACE
+    assert call(desc(), ws_bytes=8) == spiffy.EWORKSPACE
+    assert call(desc(), logits=None) == spiffy.EINVAL
+    assert call(desc(budget=11)) == spiffy.EINVAL        # more drafts kept than formulas exist
+    assert call(desc(budget=0)) == spiffy.EINVAL
+    assert call(desc(top_k=5)) == spiffy.EUNSUPPORTED
+    assert call(desc(top_k=0)) == spiffy.EINVAL
+    assert call(desc(block_len=65)) == spiffy.EUNSUPPORTED
+    assert call(desc(row_stride=1028)) == spiffy.EINVAL
+    assert call(desc(parent_cap=0)) == spiffy.EINVAL
+    assert lib.spiffy_draft_blocks_workspace(ctypes.byref(desc(vocab=0))) == 0
+
+
 def test_binding_refuses_cpu_tensors():
     import torch
     t = torch.zeros(1, 1, 4, 8)
