@@ -23,6 +23,7 @@ constexpr int kThreads = 128;  // top-k kernel
 constexpr int kVecs = 8;       // 128-bit vectors per thread
 constexpr int kMaxK = 4;       // vocabulary ranks
 constexpr int kBuildThreads = 1024;  // a warp per block position
+constexpr int kGraphInts = 6144;     // shared-memory copy of the draft graph (24 KB)
 
 struct __align__(16) TopPartial {
   float m, s;          // slice maximum, sum of exp(x - m)
@@ -208,7 +209,7 @@ __device__ bool strict_subset(const BuildArgs& g, int a, int c) {
 
 // grid = B sequences, 1024 threads; dynamic shared memory, see the carve-up below.
 __global__ void __launch_bounds__(kBuildThreads)
-draft_build_kernel(const BuildArgs g) {
+draft_build_kernel(BuildArgs g) {
 #if __CUDA_ARCH__ >= 900
   cudaGridDependencySynchronize();
 #endif
@@ -226,6 +227,23 @@ draft_build_kernel(const BuildArgs g) {
   __shared__ int n_masked;
   const int32_t* state = g.state + (int64_t)b * L;
   if (tid == 0) n_masked = 0;
+  // The formulas are walked several times with dependent reads: when the graph
+  // fits, copy it to shared memory (the copy overlaps step 1) and walk it there.
+  __shared__ int32_t graph_smem[kGraphInts];
+  {
+    const int npairs = g.formula_off[D], nkids = g.child_off[D];
+    if (2 * (D + 1) + 2 * npairs + nkids <= kGraphInts) {
+      int32_t* f_off = graph_smem;
+      int32_t* c_off = f_off + D + 1;
+      int32_t* f_i = c_off + D + 1;
+      int32_t* f_j = f_i + npairs;
+      int32_t* c_idx = f_j + npairs;
+      for (int i = tid; i <= D; i += kBuildThreads) { f_off[i] = g.formula_off[i]; c_off[i] = g.child_off[i]; }
+      for (int i = tid; i < npairs; i += kBuildThreads) { f_i[i] = g.formula_i[i]; f_j[i] = g.formula_j[i]; }
+      for (int i = tid; i < nkids; i += kBuildThreads) c_idx[i] = g.child_idx[i];
+      g.formula_off = f_off; g.child_off = c_off; g.formula_i = f_i; g.formula_j = f_j; g.child_idx = c_idx;
+    }
+  }
   __syncthreads();
 
   // 1. candidates c_ij and their probabilities: one warp per position
