@@ -74,6 +74,17 @@ cudaError_t launch_pdl(void (*kern)(Args...), dim3 grid, dim3 block, size_t smem
   return cudaLaunchKernelEx(&cfg, kern, args...);
 }
 
+// The next kernel in the stream may be launched from here on (it still waits
+// in cudaGridDependencySynchronize() for this one to finish), which takes its
+// launch latency off the critical path.  Used by the small kernels only: behind
+// the attention and the decision reduce it measured slower, their successors'
+// many CTAs crowding the SMs early.
+__device__ __forceinline__ void pdl_launch_dependents() {
+#if defined(__CUDA_ARCH__) && __CUDA_ARCH__ >= 900
+  cudaTriggerProgrammaticLaunchCompletion();
+#endif
+}
+
 inline spiffy_status check_launch() {
   return cudaGetLastError() == cudaSuccess ? SPIFFY_OK : SPIFFY_ECUDA;
 }

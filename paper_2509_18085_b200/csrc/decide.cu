@@ -240,6 +240,7 @@ decide_finalize_kernel(const Partial* __restrict__ partials, int splits, int N,
                        int32_t* __restrict__ n_unmask_out,
                        int32_t* __restrict__ dev_status) {
 #if __CUDA_ARCH__ >= 900
+  pdl_launch_dependents();
   cudaGridDependencySynchronize();  // the reduce kernel's partials are visible
 #endif
   const int node = blockIdx.x;

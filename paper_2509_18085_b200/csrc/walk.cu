@@ -16,6 +16,7 @@ accept_walk_kernel(int N, int L, const int32_t* __restrict__ block_tokens,
                    int32_t* __restrict__ next_block,
                    int32_t* __restrict__ dev_status, int stage_in_smem) {
 #if __CUDA_ARCH__ >= 900
+  pdl_launch_dependents();
   cudaGridDependencySynchronize();  // the decision kernel's outputs are visible
 #endif
   const int b = blockIdx.x;
