@@ -4,27 +4,32 @@
 // Work decomposition.  For one sequence b and one key/value head g, the query
 // rows are all (node n, position l, query head of the group) triples; they all
 // read the same P context keys, and a row of node n additionally reads the L
-// keys of node n's own block.  A CTA owns one M-tile: TNL consecutive (n, l)
-// positions times the `group` query heads of g (TNL = 128 / group, so at most
-// 128 rows), and walks over key tiles of 128 keys: first the context tiles,
+// keys of node n's own block.  An M-tile is TNL consecutive (n, l) positions
+// times the `group` query heads of g (TNL = 128 / group, so at most 128 rows);
+// a CTA owns one M-tile, or two neighbouring ones (see the kernel), and walks
+// over key tiles of 128 keys: first the context tiles,
 // then the tiles covering the block keys of the nodes its rows belong to.  The
 // mask is never materialised: a context tile is visible to every row, and in a
 // block-key tile row r sees exactly the columns of its own node, a contiguous
 // column range computed from indices.
 //
 // Pipeline inside a CTA (320 threads):
-//   warp 0      TMA producer: Q once, then K and V tiles into two 3-stage rings
+//   warp 0      TMA producer: Q once, then K and V tiles into two rings (seven
+//               32 KB tiles of shared memory in all)
 //   warp 1      allocates tensor memory; one lane issues tcgen05.mma:
 //               S = Q K^T (fp32 in TMEM, double buffered), O += P V
-//   warps 2-9   two softmax warpgroups; the first takes the even key tiles, the
-//               second the odd ones, each with its own S buffer, accumulator O
-//               and running (maximum, sum), so that the exponentials of one
-//               tile overlap the other tile's products.  One thread per row
+//   warps 2-9   two softmax warpgroups, each with its own S buffer, accumulator
+//               O and running (maximum, sum), so that the exponentials of one
+//               tile overlap the other tile's products: with one M-tile per
+//               CTA the first takes the even key tiles and the second the odd
+//               ones (a CTA with few key tiles leaves it all to the first);
+//               with two M-tiles each warpgroup owns one.  One thread per row
 //               reads S from TMEM, writes P (bf16) back over it as the A
 //               operand of the second product, and rescales its O only when
 //               the maximum grew by more than 2^8 (exact: O and the sum always
-//               share one reference maximum).  At the end the two accumulators
-//               are merged, normalised and stored.
+//               share one reference maximum).  At the end the accumulators
+//               are merged where two belong to the same rows, normalised and
+//               stored.
 // With several splits (grid.z) each CTA handles a slice of the key tiles and
 // stores an unnormalised partial (O, reference maximum, sum); a second kernel
 // merges the partials.
