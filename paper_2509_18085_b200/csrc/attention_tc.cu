@@ -84,6 +84,7 @@ struct Params {
   int MT;       // M-tiles per (sequence, kv head)
   int TP;       // context key tiles
   int splits;
+  int pair;  // the two splits are the two CTAs of a cluster and merge through shared memory
   float scale_log2;
   __nv_bfloat16* out;
   float* part_o;   // [splits][B*Hkv][MT][128][128]
@@ -468,7 +469,9 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
           pml[1] = l_run;
         }
       }
-    } else if (!(solo && wg == 1)) {
+    } else {
+    const bool active = !(solo && wg == 1);
+    const bool pair = p.pair != 0;
     float m_o = m_alt, l_o = l_alt;  // state of the other buffer
     if (!solo) {
       constexpr uint32_t kColMl = BN / 2;  // first S column that no P lies over
@@ -491,35 +494,85 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     const float w_a = has_a ? ex2(m_a - m_all) : 0.f;
     const float w_b = has_b ? ex2(m_b - m_all) : 0.f;
     const float l_all = w_a * l_a + w_b * l_b;
-    if (ok) {
-      const float inv = p.splits == 1 ? 1.0f / l_all : 1.0f;
-      const float f_a = w_a * inv, f_b = w_b * inv;
-      const int64_t tile = ((int64_t)split * gridDim.y + bg) * p.MT + mt;
-      __nv_bfloat16* dst =
-          p.out + (((int64_t)b * p.NL + nl) * p.Hq + (int64_t)g * p.group + hh) * HD;
-      float* po = p.part_o + (tile * BM + r) * HD;
+    // 32 columns of this CTA's two accumulators, merged against m_all and scaled by f
+    auto merged = [&](int c0, float f, float (&o)[32]) {
+      uint32_t oa[32], ob[32];
+      tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + c0), oa);
+      tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + HD + c0), ob);
+      const float f_a = w_a * f, f_b = w_b * f;
 #pragma unroll
+      for (int c = 0; c < 32; ++c)
+        o[c] = (has_a ? __uint_as_float(oa[c]) * f_a : 0.f) +
+               (has_b ? __uint_as_float(ob[c]) * f_b : 0.f);
+    };
+    auto store_bf16 = [&](__nv_bfloat16* at, const float (&o)[32]) {
+#pragma unroll
+      for (int c = 0; c < 32; c += 8) {
+        uint4 w;
+        w.x = pack_bf16(o[c], o[c + 1]);
+        w.y = pack_bf16(o[c + 2], o[c + 3]);
+        w.z = pack_bf16(o[c + 4], o[c + 5]);
+        w.w = pack_bf16(o[c + 6], o[c + 7]);
+        *reinterpret_cast<uint4*>(at + c) = w;
+      }
+    };
+    __nv_bfloat16* dst =
+        p.out + (((int64_t)b * p.NL + nl) * p.Hq + (int64_t)g * p.group + hh) * HD;
+    if (pair) {
+      // The other half of the key tiles went to the peer CTA of the cluster.  Each of the
+      // two finishes 64 of the 128 columns: it sends its partial of the peer's columns
+      // into the peer's shared memory (the Q tile, idle by then) and merges what it gets.
+      const uint32_t rank = (uint32_t)split, peer = rank ^ 1u;
+      const int cc0 = solo ? 0 : wg, cc1 = solo ? 2 : wg + 1;  // 32-column chunks of a half
+      cluster_sync_all();  // both CTAs have finished their products: Q and K tiles are idle
+      if (active && ok) {
+        tc_fence_after_sync();
+        const uint32_t q_peer = map_to_cta(smem_u32(sq), peer);
+        for (int cc = cc0; cc < cc1; ++cc) {
+          float o[32];
+          merged(64 * (int)peer + 32 * cc, 1.0f, o);
+#pragma unroll
+          for (int k = 0; k < 8; ++k)  // 16-byte chunk (8 cc + k) of row r: chunk-major, rows contiguous
+            st_cluster_f4(q_peer + (uint32_t)(8 * cc + k) * 2048u + (uint32_t)r * 16u, o[4 * k],
+                          o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
+        }
+        if (solo || wg == 0) st_cluster_f2(map_to_cta(smem_u32(sk), peer) + (uint32_t)r * 8u, m_all, l_all);
+      }
+      cluster_sync_all();  // the peer's partial has arrived
+      if (active && ok) {
+        const float2 mlp = *reinterpret_cast<const float2*>(sk + r * 8);
+        const float m_p = mlp.x, l_p = mlp.y;
+        const float m_fin = fmaxf(m_all, m_p);
+        const float w_l = m_all != -INFINITY ? ex2(m_all - m_fin) : 0.f;
+        const float w_p = m_p != -INFINITY ? ex2(m_p - m_fin) : 0.f;
+        const float inv = 1.0f / (w_l * l_all + w_p * l_p);
+        for (int cc = cc0; cc < cc1; ++cc) {
+          float o[32];
+          merged(64 * (int)rank + 32 * cc, w_l * inv, o);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const float4 q4 = *reinterpret_cast<const float4*>(sq + (8 * cc + k) * 2048 + r * 16);
+            if (w_p != 0.f) {
+              o[4 * k] += q4.x * (w_p * inv);
+              o[4 * k + 1] += q4.y * (w_p * inv);
+              o[4 * k + 2] += q4.z * (w_p * inv);
+              o[4 * k + 3] += q4.w * (w_p * inv);
+            }
+          }
+          if (row_ok) store_bf16(dst + 64 * (int)rank + 32 * cc, o);
+        }
+      }
+    } else if (active && ok) {
+      const float inv = p.splits == 1 ? 1.0f / l_all : 1.0f;
+      const int64_t tile = ((int64_t)split * gridDim.y + bg) * p.MT + mt;
+      float* po = p.part_o + (tile * BM + r) * HD;
       // solo: all 128 columns; otherwise each warpgroup stores one half
       for (int c0 = solo ? 0 : wg * 64; c0 < (solo ? HD : wg * 64 + 64); c0 += 32) {
-        uint32_t oa[32], ob[32];
-        tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + c0), oa);
-        tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + HD + c0), ob);
         float o[32];
-#pragma unroll
-        for (int c = 0; c < 32; ++c)
-          o[c] = (has_a ? __uint_as_float(oa[c]) * f_a : 0.f) +
-                 (has_b ? __uint_as_float(ob[c]) * f_b : 0.f);
+        merged(c0, inv, o);
         if (row_ok) {
           if (p.splits == 1) {
-#pragma unroll
-            for (int c = 0; c < 32; c += 8) {
-              uint4 w;
-              w.x = pack_bf16(o[c], o[c + 1]);
-              w.y = pack_bf16(o[c + 2], o[c + 3]);
-              w.z = pack_bf16(o[c + 4], o[c + 5]);
-              w.w = pack_bf16(o[c + 6], o[c + 7]);
-              *reinterpret_cast<uint4*>(dst + c0 + c) = w;
-            }
+            store_bf16(dst + c0, o);
           } else {
 #pragma unroll
             for (int c = 0; c < 32; c += 4)
@@ -536,6 +589,10 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     }  // NQ == 1
   }
 
+  if (NQ == 1 && p.pair && (warp < 2 || T <= 0)) {
+    cluster_sync_all();  // the two barriers of the paired epilogue
+    cluster_sync_all();
+  }
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) {
@@ -618,7 +675,8 @@ bool make_map(CUtensorMap* m, const void* base, int heads, int64_t rows, int out
 
 struct Plan {
   int group, TNL, NL, MT, TP, splits;
-  int nq;  // M-tiles per CTA
+  int nq;    // M-tiles per CTA
+  int pair;  // key tiles split over the two CTAs of a cluster (no workspace, no merge kernel)
   int64_t tiles;  // B * Hkv * MT
 };
 
@@ -634,12 +692,17 @@ Plan make_plan(const spiffy_attn_desc& d) {
   // tile then serves twice as many rows per trip from L2.
   pl.nq = ((int64_t)d.batch * d.n_kv_heads * ((pl.MT + 1) / 2) >= 148) ? 2 : 1;
   // Fewer CTAs than SMs: cut the key tiles of each M-tile into slices so that
-  // the context streams through more SMs at once.
+  // the context streams through more SMs at once.  Many slices go through the
+  // workspace and a merge kernel (which costs about three key tiles); two
+  // slices are the two CTAs of a cluster and merge through shared memory.
   int splits = 1;
-  if (pl.tiles < 120 && pl.TP + 1 >= 8) {  // a merge pass costs about three key tiles
+  pl.pair = 0;
+  if (pl.tiles < 120 && pl.TP + 1 >= 8 && 148 / pl.tiles >= 3) {
     splits = (int)(148 / pl.tiles);
     if (splits > pl.TP + 1) splits = pl.TP + 1;
-    if (splits < 1) splits = 1;
+  } else if (pl.nq == 1 && 2 * pl.tiles <= 148 && pl.TP + 1 >= 4) {
+    splits = 2;
+    pl.pair = 1;
   }
   pl.splits = splits;
   return pl;
@@ -657,7 +720,7 @@ bool attention_tc_supported(const spiffy_attn_desc& d) {
 
 size_t attention_tc_workspace_bytes(const spiffy_attn_desc& d) {
   const Plan pl = make_plan(d);
-  if (pl.splits == 1) return 0;
+  if (pl.splits == 1 || pl.pair) return 0;
   return (size_t)pl.splits * pl.tiles * BM * (HD + 2) * sizeof(float);
 }
 
@@ -682,6 +745,7 @@ spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q, cons
   p.B = d.batch; p.N = d.n_nodes; p.L = d.block_len; p.P = d.prefix_len;
   p.Hq = d.n_q_heads; p.Hkv = d.n_kv_heads; p.group = pl.group;
   p.TNL = pl.TNL; p.NL = pl.NL; p.MT = pl.MT; p.TP = pl.TP; p.splits = pl.splits;
+  p.pair = pl.pair;
   const float scale = d.scale != 0.f ? d.scale : 1.0f / sqrtf((float)d.head_dim);
   p.scale_log2 = scale * kLog2e;
   p.out = static_cast<__nv_bfloat16*>(out);
@@ -696,11 +760,26 @@ spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q, cons
     return SPIFFY_ECUDA;
   const dim3 grid((pl.MT + pl.nq - 1) / pl.nq, d.batch * d.n_kv_heads, pl.splits);
   auto kern = pl.nq == 2 ? graph_attention_tc_kernel<2> : graph_attention_tc_kernel<1>;
-  if (launch_pdl(kern, grid, dim3(kThreads), (size_t)kSmemBytes, stream, tm_q, tm_kp, tm_vp, tm_kb,
-                 tm_vb, p) != cudaSuccess)
-    return SPIFFY_ECUDA;
+  {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;  // pairs along grid.z, only when asked for
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 2;
+    cfg.attrs = attr;
+    cfg.numAttrs = pl.pair ? 2 : 1;
+    if (cudaLaunchKernelEx(&cfg, kern, tm_q, tm_kp, tm_vp, tm_kb, tm_vb, p) != cudaSuccess)
+      return SPIFFY_ECUDA;
+  }
   count_launch();
-  if (pl.splits > 1) {
+  if (pl.splits > 1 && !pl.pair) {
     const int64_t rows = (int64_t)d.batch * pl.NL * d.n_q_heads;
     if (launch_pdl(graph_attention_combine_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256),
                    (size_t)0, stream, p) != cudaSuccess)
