@@ -181,14 +181,17 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
+  if (threadIdx.x == 0) {  // the descriptors are kernel parameters: fetch them ahead of the wait
+    prefetch_tensormap(&tm_q);
+    prefetch_tensormap(p.TP > 0 ? &tm_kp : &tm_kb);
+    prefetch_tensormap(p.TP > 0 ? &tm_vp : &tm_vb);
+  }
   // everything above is on-chip set-up; global memory is touched from here on
   cudaGridDependencySynchronize();
 
   if (warp == 0) {
     // ------------------------------------------------------------ producer --
     if (lane == 0 && T > 0) {
-      prefetch_tensormap(&tm_q);
-      prefetch_tensormap(p.TP > 0 ? &tm_kp : &tm_kb);
       mbar_arrive_expect_tx(q_full, (uint32_t)NQ * 2u * rows_box * 128u);
 #pragma unroll
       for (int q = 0; q < NQ; ++q) {  // an M-tile beyond the last one reads as zeros
