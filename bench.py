@@ -478,10 +478,10 @@ def main():
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
-        sec, what = oracle_step_time(cfg, work[0], 5)
+        sec, what = oracle_step_time(cfg, work[0], 80)  # about ten seconds of CPU work
         line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": oracle.max_threads(),
                                 "kind": "oracle",
-                                "sample": f"median of 5 full steps of the same workload ({what})"}
+                                "sample": f"median of 80 full steps of the same workload ({what})"}
     if rank == 0:
         print(json.dumps(line))
     replicas.finish(ranks)
