@@ -15,7 +15,9 @@
  *                            App. A) evaluated for every node of the graph;
  *   spiffy_accept_walk       step 5 of Algorithm 1: the walk through the draft
  *                            graph (Sec. 4.4.1, Eqs. draft-graph-1..3) to the
- *                            deepest accepted node.
+ *                            deepest accepted node;
+ *   spiffy_draft_blocks      drafting and pruning (Sec. 4.4.2, Sec. 4.4.4): the
+ *                            draft blocks and parent lists of the next step.
  *
  * Vocabulary (paper notation in brackets where it differs):
  *   B  batch of independent sequences            N  nodes of the draft graph,
@@ -33,7 +35,8 @@
  *     NULL = the default stream) and never synchronise the device.
  *   - Scratch memory is caller-provided: size it with the *_workspace() query.
  *     Its contents on entry are arbitrary; calls sharing one workspace must be
- *     ordered on one stream.
+ *     ordered on one stream.  (spiffy_unmask_decide_static is the exception: it
+ *     keeps its scratch inside the library.)
  *   - Tensor base addresses must be 16-byte aligned, else SPIFFY_EINVAL.
  *   - Host-detectable problems return a status code and launch nothing.
  *     Device-detectable problems set bits in a caller-provided status word and
