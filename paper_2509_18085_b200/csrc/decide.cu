@@ -267,12 +267,12 @@ decide_finalize_kernel(const Partial* __restrict__ partials, int splits, int N,
     }
     if (sub == 0 && pos < L) {
       const bool masked = state == mask_id;
-      const float conf = masked ? 1.0f / s : -INFINITY;
+      const float conf = masked ? fminf(1.0f, 1.0f / s) : -INFINITY;  // the sum can round just below one
       conf_out[row] = conf;
       tok_out[row] = masked ? idx : state;
       sconf[pos] = conf;
-      // a usable row has a finite maximum and a finite sum of at least one
-      if (masked && (!(fabsf(m) < INFINITY) || !(s >= 1.0f) || !(s < INFINITY))) {
+      // a usable row has a finite maximum and a finite, positive sum (the sum is one or more up to rounding)
+      if (masked && (!(fabsf(m) < INFINITY) || !(s > 0.f) || !(s < INFINITY))) {
         if (dev_status) atomicOr(dev_status + node / N, SPIFFY_DEV_NONFINITE);
       }
     }

@@ -268,7 +268,7 @@ draft_build_kernel(BuildArgs g) {
       s = s * ((m == M) ? 1.f : ex2((m - M) * kLog2e)) + s2 * ((m2 == M) ? 1.f : ex2((m2 - M) * kLog2e));
       m = M;
     }
-    if (lane == 0 && (!(fabsf(m) < INFINITY) || !(s >= 1.0f) || !(s < INFINITY)) && g.dev_status)
+    if (lane == 0 && (!(fabsf(m) < INFINITY) || !(s > 0.f) || !(s < INFINITY)) && g.dev_status)
       atomicOr(g.dev_status + b, SPIFFY_DEV_NONFINITE);
     // the K best of the splits * K slice candidates (value desc, id asc): every lane
     // first sorts the candidates it reads (each is read once), then K rounds pick the

@@ -120,3 +120,21 @@ def test_full_size_long_batched_sampled_nodes():
                                       w.k_block[b:b + 1, n:n + 1], w.v_block[b:b + 1, n:n + 1])
         assert np.max(np.abs(got[b, n] - want[0, 0])) <= G.TOL["bf16"]
     assert np.all(np.isfinite(got))
+
+
+@pytest.mark.parametrize("kernel", [spiffy.ATTN_SIMT, spiffy.ATTN_TCGEN05])
+def test_peaked_scores_and_a_late_maximum(kernel):
+    """Scores far from zero, and a row maximum that only shows up in the last key
+    tiles: the accumulator is rescaled late (the reference maximum moves by far
+    more than its slack) and probabilities are nearly one-hot."""
+    cfg = W.config(2, n_nodes=3, prefix_len=700)
+    w = W.make(cfg, 21, decision=False)
+    w.q *= 6.0                       # scores of standard deviation 6 before the softmax
+    w.k_prefix[:, 600:650] *= 3.0    # the largest scores sit late in the context ...
+    w.k_block[:, 1] *= 4.0           # ... or in one node's own block
+    for a in ("q", "k_prefix", "k_block"):
+        setattr(w, a, W.round_to(getattr(w, a), "bf16"))
+    got = G.gpu_attention(w, kernel)
+    want = oracle_attention(w)
+    assert np.all(np.isfinite(got))
+    assert np.max(np.abs(got - want)) <= G.TOL["bf16"]

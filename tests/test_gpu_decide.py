@@ -185,3 +185,25 @@ def test_walk_flags_malformed_parent_lists():
                                   G.to_dev(bits))
     assert g.dev_status.cpu().tolist() == [0, spiffy.DEV_BADGRAPH]
     assert g.accepted_node.cpu().tolist() == [0, 0]
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_wide_logit_range(dtype):
+    """Logits spread over +-80 with the row maximum anywhere in the row: the sums
+    of exponentials must neither overflow nor lose the small terms' order."""
+    V = 40000
+    cfg, logits, tokens = small_case(1, 2, 8, V, dtype, seed=5, p_unmasked=0.0)
+    r = np.random.default_rng(6)
+    logits *= 8.0
+    for l in range(8):
+        logits[0, 0, l, int(r.integers(0, V - 1))] = 80.0 - l   # one dominant token per row
+        logits[0, 1, l, int(r.integers(0, V - 1))] = -80.0      # a far-away minimum changes nothing
+    logits = W.round_to(logits, dtype)
+    dec = spiffy.spiffy_unmask_decide(G.to_dev(logits, G.tdtype(cfg)), G.to_dev(tokens), cfg.mask_id,
+                                      spiffy.RULE_THRESHOLD, 1, 0.9)
+    o = oracle.unmask_decide(logits, tokens, cfg.mask_id, oracle.RULE_THRESHOLD, 1, 0.9)
+    assert np.array_equal(dec.top_tok.cpu().numpy(), o.top_tok)
+    np.testing.assert_allclose(dec.conf.cpu().numpy(), o.conf, atol=G.TOL[dtype])
+    safe = o.margin >= 1e-3
+    assert np.array_equal(G.bits_np(dec.unmask_bits)[safe], o.unmask_bits[safe])
+    assert int(dec.dev_status.cpu().sum()) == 0
