@@ -60,6 +60,8 @@ def test_configs(index, n_nodes, kernel):
     dict(batch=1, n_nodes=5, block_len=16, prefix_len=0, n_q_heads=4, n_kv_heads=4, head_dim=128),
     dict(batch=2, n_nodes=7, block_len=32, prefix_len=300, n_q_heads=8, n_kv_heads=2, head_dim=128),
     dict(batch=1, n_nodes=9, block_len=8, prefix_len=1000, n_q_heads=3, n_kv_heads=3, head_dim=128),
+    # 26 nodes of 5 positions under one M-tile: their block keys need two key tiles
+    dict(batch=1, n_nodes=30, block_len=5, prefix_len=70, n_q_heads=2, n_kv_heads=2, head_dim=128),
     # enough M-tiles for the two-tiles-per-CTA variant; an odd tile count leaves one CTA half empty
     dict(batch=3, n_nodes=9, block_len=32, prefix_len=300, n_q_heads=32, n_kv_heads=32, head_dim=128),
     dict(batch=10, n_nodes=6, block_len=16, prefix_len=130, n_q_heads=32, n_kv_heads=16, head_dim=128),

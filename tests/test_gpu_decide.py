@@ -207,3 +207,29 @@ def test_wide_logit_range(dtype):
     safe = o.margin >= 1e-3
     assert np.array_equal(G.bits_np(dec.unmask_bits)[safe], o.unmask_bits[safe])
     assert int(dec.dev_status.cpu().sum()) == 0
+
+
+def test_degenerate_shapes():
+    """A graph without drafts, a block of one position, uniform rows and a tiny vocabulary."""
+    # N = 1, L = 1: the walk has nowhere to go
+    logits = np.zeros((2, 1, 1, 16), dtype=np.float32)
+    logits[0, 0, 0, 5] = 3.0
+    tokens = np.full((2, 1, 1), 15, dtype=np.int32)
+    dec = spiffy.spiffy_unmask_decide(G.to_dev(logits), G.to_dev(tokens), 15, spiffy.RULE_TOPS)
+    o = oracle.unmask_decide(logits, tokens, 15, oracle.RULE_TOPS)
+    assert dec.top_tok.cpu().numpy().tolist() == [[[5]], [[0]]]       # uniform row: lowest token id
+    np.testing.assert_allclose(dec.conf.cpu().numpy(), o.conf, atol=1e-6)
+    assert abs(float(dec.conf[1, 0, 0]) - 1.0 / 16) < 1e-6
+    off = np.zeros((2, 2), dtype=np.int32)
+    idx = np.zeros((2, 4), dtype=np.int32)
+    walk = spiffy.spiffy_accept_walk(G.to_dev(tokens), G.to_dev(off), G.to_dev(idx), dec.top_tok, dec.unmask_bits)
+    assert walk.accepted_node.cpu().tolist() == [0, 0] and walk.n_accepted.cpu().tolist() == [0, 0]
+    assert walk.next_block.cpu().numpy().tolist() == [[5], [0]]
+    # V = 4 (half a 128-bit vector of fp32... one vector exactly), every position unmasked in node 1
+    logits = np.arange(2 * 3 * 4, dtype=np.float32).reshape(1, 2, 3, 4) % 5
+    tokens = np.array([[[3, 3, 1], [0, 1, 2]]], dtype=np.int32)
+    dec = spiffy.spiffy_unmask_decide(G.to_dev(logits), G.to_dev(tokens), 3, spiffy.RULE_THRESHOLD, 1, 0.5)
+    o = oracle.unmask_decide(logits, tokens, 3, oracle.RULE_THRESHOLD, 1, 0.5)
+    assert np.array_equal(dec.top_tok.cpu().numpy(), o.top_tok)
+    assert np.array_equal(G.bits_np(dec.unmask_bits), o.unmask_bits)
+    assert dec.n_unmask.cpu().numpy().tolist() == o.n_unmask.tolist() and o.n_unmask[0, 1] == 0

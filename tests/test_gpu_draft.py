@@ -102,3 +102,17 @@ def test_drafts_feed_the_walk():
     walk = spiffy.spiffy_accept_walk(d.tokens, d.parent_off, d.parent_idx, G.to_dev(top), G.to_dev(bits))
     assert walk.accepted_node.cpu().tolist() == [node] and walk.n_accepted.cpu().tolist() == [1]
     assert int(walk.dev_status.cpu().sum()) == 0
+
+
+def test_nothing_left_to_draft_and_single_rank():
+    """A fully unmasked block yields no draft; top_k = 1 and budget = D keep every buildable formula."""
+    V, L = 64, 4
+    r = np.random.default_rng(3)
+    logits = (r.standard_normal((2, L, V)) * 2).astype(np.float32)
+    state = np.array([[1, 2, 3, 4], [V - 1, V - 1, 7, V - 1]], dtype=np.int32)
+    formulas = [[(0, 0)], [(1, 0)], [(0, 0), (1, 0)], [(0, 0), (1, 0), (2, 0)], [(3, 0)]]
+    children = [[2], [2], [3], [], []]
+    got, want = run_both(logits, state, V - 1, 5, 1, torch.float32, formulas, children)
+    assert_parity(got, want)
+    assert got.kept[0].cpu().tolist() == [-1] * 5 and got.kept[1].cpu().tolist() == [0, 1, 2, 3, -1]
+    assert torch.equal(got.tokens[0], torch.from_numpy(state[0]).cuda().expand(6, L))
