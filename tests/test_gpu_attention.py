@@ -60,6 +60,10 @@ def test_configs(index, n_nodes, kernel):
     dict(batch=1, n_nodes=5, block_len=16, prefix_len=0, n_q_heads=4, n_kv_heads=4, head_dim=128),
     dict(batch=2, n_nodes=7, block_len=32, prefix_len=300, n_q_heads=8, n_kv_heads=2, head_dim=128),
     dict(batch=1, n_nodes=9, block_len=8, prefix_len=1000, n_q_heads=3, n_kv_heads=3, head_dim=128),
+    # query-head groups of 16, 128 and 3 per kv head: 8, 1 and 42 (node, position) pairs per M-tile
+    dict(batch=1, n_nodes=3, block_len=10, prefix_len=50, n_q_heads=16, n_kv_heads=1, head_dim=128),
+    dict(batch=1, n_nodes=2, block_len=3, prefix_len=20, n_q_heads=128, n_kv_heads=1, head_dim=128),
+    dict(batch=2, n_nodes=4, block_len=12, prefix_len=129, n_q_heads=6, n_kv_heads=2, head_dim=128),
     # 26 nodes of 5 positions under one M-tile: their block keys need two key tiles
     dict(batch=1, n_nodes=30, block_len=5, prefix_len=70, n_q_heads=2, n_kv_heads=2, head_dim=128),
     # enough M-tiles for the two-tiles-per-CTA variant; an odd tile count leaves one CTA half empty
