@@ -152,16 +152,25 @@ def vanilla_decode(model, state0, rule, top_s=1, threshold=0.9, decide=_default_
 def speculative_decode(model, state0, drafter, rule, top_s=1, threshold=0.9,
                        decide=_default_decide, walk=_default_walk):
     """Decoding with Algorithm 1.  ``drafter(state, call_index)`` returns an
-    array [D,L] of draft blocks (possibly empty).  Returns (states visited,
-    per call the number of accepted drafts whose distribution was used)."""
+    array [D,L] of draft blocks (possibly empty).  A drafter with the attribute
+    ``uses_last_logits`` is called as ``drafter(state, call_index, logits)``
+    with the distribution [L,V] of the last node accepted by the previous call
+    (None before the first call): the distribution ``state`` was unmasked from.
+    Returns (states visited, per call the number of accepted drafts whose
+    distribution was used)."""
     mask_id = model.mask_id
     state = np.asarray(state0, dtype=np.int32).copy()
     L = state.shape[0]
     traj = [state.copy()]
     accepted = []
     call = 0
+    last_logits = None
     while np.any(state == mask_id):
-        drafts = np.asarray(drafter(state, call), dtype=np.int32).reshape(-1, L)
+        if getattr(drafter, "uses_last_logits", False):
+            drafts = drafter(state, call, last_logits)
+        else:
+            drafts = drafter(state, call)
+        drafts = np.asarray(drafts, dtype=np.int32).reshape(-1, L)
         # order drafts by how many tokens they unmask so that parents precede
         # children, and drop exact duplicates
         if len(drafts):
@@ -186,6 +195,7 @@ def speculative_decode(model, state0, drafter, rule, top_s=1, threshold=0.9,
             traj.append(np.where(sel, top_tok[0, node], states[node]).astype(np.int32))
         assert np.array_equal(traj[-1], next_block[0])
         state = next_block[0].astype(np.int32).copy()
+        last_logits = np.asarray(logits)[0, int(path[0][int(hops[0])])]
         # an accepted draft saves a model call only when its distribution is
         # used, i.e. when it still had something to unmask
         accepted.append(sum(1 for node in path[0][1: int(hops[0]) + 1]
@@ -263,4 +273,28 @@ def auto_drafter(model, formulas, children, budget, top_k, draft=None):
                        model.mask_id)
         return np.asarray(tokens)[0, 1:]
 
+    return drafter
+
+
+def carry_over_drafter(mask_id, formulas, children, budget, top_k, draft=None):
+    """Auto-speculation without any extra model call: the drafts of a call are
+    built from the distribution of the last node accepted by the previous call
+    (Algorithm 1 hands that distribution on; Sec. 4.4.2 drafts from the
+    distribution at hand), with the ranks taken over the positions still masked
+    in the new current block.  The first call has no distribution yet and
+    carries no drafts."""
+    from . import drafting
+
+    def default_draft(logits, state, mask):
+        return drafting.draft_blocks(logits, state, mask, formulas, children, budget, top_k).tokens
+
+    build = draft or default_draft
+
+    def drafter(state, call, logits):
+        if logits is None:
+            return np.zeros((0, len(state)), dtype=np.int32)
+        tokens = build(np.ascontiguousarray(logits[None], dtype=np.float32), state[None].astype(np.int32), mask_id)
+        return np.asarray(tokens)[0, 1:]
+
+    drafter.uses_last_logits = True
     return drafter

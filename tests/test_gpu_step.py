@@ -154,3 +154,49 @@ def test_auto_speculation_through_the_cuda_drafting_call():
         assert model.calls == calls - sum(accepted)
         saved += sum(accepted)
     assert saved > 0
+
+
+def test_calibrated_graph_with_carried_over_distribution_on_the_cuda_path():
+    """Offline calibration (Algorithm 2) on plain runs, then decoding where every
+    call's drafts are built by spiffy_draft_blocks from the distribution of the
+    last node the previous call accepted: no extra model call, the trajectory is
+    plain decoding's (App. A) and the calibrated graph saves calls."""
+    from paper_2509_18085_b200 import calibration
+
+    def prompt(seed):
+        model = toy.ToyModel(seed=7, sharpness=3.0)
+        r = np.random.default_rng(seed)
+        start = np.full(model.block_len, model.mask_id, dtype=np.int32)
+        known = r.choice(model.block_len, size=2, replace=False)
+        start[known] = r.integers(0, model.vocab - 1, size=2)
+        return model, start
+
+    _, decide, walk = gpu_backends()
+    sequences = []
+    for seed in range(10):
+        model, start = prompt(seed)
+        states = toy.vanilla_decode(model, start, oracle.RULE_TOPS, decide=decide)
+        logits = [model(s[None])[0, 0] for s in states[:-1]]
+        sequences += calibration.record(states[1:], logits[:-1], model.mask_id, 3, 3)
+    formulas, children, _ = calibration.calibrate(calibration.build_graph(sequences, 3), 6)
+    assert len(formulas) == 6
+    graph = spiffy.draft_graph(formulas, children)
+
+    def draft(logits, state, mask_id):
+        d = spiffy.spiffy_draft_blocks(G.to_dev(logits), G.to_dev(state), mask_id, graph, len(formulas), 3)
+        assert int(d.dev_status.max().item()) == 0
+        return d.tokens.cpu().numpy()
+
+    saved = steps = 0
+    for seed in range(100, 106):
+        model, start = prompt(seed)
+        vanilla = toy.vanilla_decode(model, start, oracle.RULE_TOPS, decide=decide)
+        calls = model.calls
+        model.calls = 0
+        drafter = toy.carry_over_drafter(model.mask_id, formulas, children, len(formulas), 3, draft=draft)
+        traj, accepted = toy.speculative_decode(model, start, drafter, oracle.RULE_TOPS, decide=decide, walk=walk)
+        assert len(traj) == len(vanilla) and all(np.array_equal(a, b) for a, b in zip(traj, vanilla))
+        assert model.calls == calls - sum(accepted)
+        saved += sum(accepted)
+        steps += len(vanilla) - 1
+    assert saved >= steps // 5
