@@ -21,6 +21,12 @@ smaller sorted (i, j) list; the "top in-edges" of Part 2 add no edge beyond the
 subset edges and are not modelled; a token whose rank cannot be named (its
 position was already unmasked at t, or its vocabulary rank is beyond max_rank)
 ends the look-ahead of that timestep.
+
+Pins (tests/test_oracle_calibration.py): a three-position run worked by hand
+(ranks, sequences, counts, ties); a nine-node graph whose most frequent node has
+no parent (App. D.1) for D = 1..9; under top-S decoding the level-1 node is the
+S most confident positions with their best tokens; the closed loop on the toy
+model (the calibrated graph is accepted, a graph of deep ranks is not).
 """
 from __future__ import annotations
 
