@@ -12,8 +12,9 @@ acceptance walk (step 5).  The metric is verify steps per second.
             rotates over several distinct input sets (together larger than
             L2), timed with CUDA events on the launching stream.
 `e2e`     : the same step driven from pinned host memory through
-            VerifyStep.run_host (host-to-device copies of every input and the
-            device-to-host read of the verdict inside the timed region).
+            VerifyStep.run_host (host-to-device copies of everything the step
+            reads -- of the logits, the rows of still-masked positions -- and
+            the device-to-host read of the verdict inside the timed region).
 `roofline`: the dominant kernel (the decision reduce) against the measured HBM
             copy bandwidth; its duration comes from a second pass that replays
             the decision call alone over the same rotation of input sets.

@@ -9,6 +9,7 @@ and copies the verdict back -- the end-to-end call.
 """
 from __future__ import annotations
 
+import ctypes
 from dataclasses import dataclass
 
 import torch
@@ -52,6 +53,22 @@ def inputs_from_workload(w, device="cuda", pin=False) -> StepInputs:
     return StepInputs(mv(w.q, dt), mv(w.k_prefix, dt), mv(w.v_prefix, dt), mv(w.k_block, dt),
                       mv(w.v_block, dt), mv(w.logits, dt), mv(w.block_tokens), mv(w.parent_off),
                       mv(w.parent_idx))
+
+
+_CUDART = None
+
+
+def _cudart():
+    """The CUDA runtime torch has loaded, for row-run copies without a tensor
+    slice per run."""
+    global _CUDART
+    if _CUDART is None:
+        major = torch.version.cuda.split(".")[0]
+        _CUDART = ctypes.CDLL(f"libcudart.so.{major}")
+        _CUDART.cudaMemcpyAsync.restype = ctypes.c_int
+        _CUDART.cudaMemcpyAsync.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int,
+                                            ctypes.c_void_p]
+    return _CUDART
 
 
 class VerifyStep:
@@ -112,13 +129,34 @@ class VerifyStep:
         self.decide(x)
         return self.accept(x)
 
+    @staticmethod
+    def _masked_row_runs(host: StepInputs, mask_id: int):
+        """[start, stop) runs of logit rows whose position is still masked: the
+        only rows the decision step reads (Algorithm 1 ranks masked positions)."""
+        m = (host.block_tokens.reshape(-1) == mask_id).to(torch.int8)
+        edges = torch.diff(m, prepend=m.new_zeros(1), append=m.new_zeros(1)).nonzero().reshape(-1).tolist()
+        return list(zip(edges[0::2], edges[1::2]))
+
     def run_host(self, host: StepInputs):
         """End to end from pinned host memory: copy the step's inputs in, run
-        it, read the verdict (accepted node, hop count, next block) back."""
+        it, read the verdict (accepted node, hop count, next block) back.  Of
+        the logits only the rows of still-masked positions cross the bus (runs
+        of neighbouring rows in one copy each); the staging rows of unmasked
+        positions keep whatever they held and no kernel reads them."""
         if self.staging is None:
             self.staging = StepInputs(*[torch.empty_like(t, device=self.device) for t in host.tensors()])
+        row = host.logits.shape[-1] * host.logits.element_size()
+        base_dst, base_src = self.staging.logits.data_ptr(), host.logits.data_ptr()
+        stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+        copy = _cudart().cudaMemcpyAsync
+        for a, b in self._masked_row_runs(host, self.cfg.mask_id):
+            rc = copy(ctypes.c_void_p(base_dst + a * row), ctypes.c_void_p(base_src + a * row),
+                      ctypes.c_size_t((b - a) * row), 1, stream)  # 1 = host to device
+            if rc != 0:
+                raise RuntimeError(f"cudaMemcpyAsync failed with error {rc}")
         for dst, src in zip(self.staging.tensors(), host.tensors()):
-            dst.copy_(src, non_blocking=True)
+            if src is not host.logits:
+                dst.copy_(src, non_blocking=True)
         w = self.run(self.staging)
         for dst, src in zip(self.verdict_host, (w.accepted_node, w.n_accepted, w.next_block)):
             dst.copy_(src, non_blocking=True)
@@ -126,7 +164,11 @@ class VerifyStep:
         return self.verdict_host
 
     def h2d_bytes(self, host: StepInputs) -> int:
-        return host.nbytes()
+        """Bytes ``run_host`` copies to the device for this input."""
+        rows = sum(b - a for a, b in self._masked_row_runs(host, self.cfg.mask_id))
+        V = host.logits.shape[-1]
+        return host.nbytes() - host.logits.numel() * host.logits.element_size() \
+            + rows * V * host.logits.element_size()
 
     def d2h_bytes(self) -> int:
         return sum(t.numel() * t.element_size() for t in self.verdict_host)

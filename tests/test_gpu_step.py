@@ -200,3 +200,31 @@ def test_calibrated_graph_with_carried_over_distribution_on_the_cuda_path():
         saved += sum(accepted)
         steps += len(vanilla) - 1
     assert saved >= steps // 5
+
+
+@pytest.mark.parametrize("config", [1, 2])
+def test_end_to_end_call_from_host_memory(config):
+    """run_host copies, of the logits, only the rows of still-masked positions:
+    with every other staging row poisoned the verdict still equals the oracle's
+    and the byte count it reports is what crossed the bus."""
+    from paper_2509_18085_b200.step import VerifyStep, inputs_from_workload
+    cfg = W.config(config)
+    w = W.make(cfg, W.seed_for(config, 7))
+    host = inputs_from_workload(w, device="cpu", pin=True)
+    step = VerifyStep(cfg)
+    step.run_host(host)  # allocates the staging buffers
+    step.staging.logits.fill_(float("nan"))
+    acc, hops, nxt = [t.clone() for t in step.run_host(host)]
+    odec, owalk = G.oracle_decide(w)
+    n = G.assert_decision_parity(w, step.decision, step.walk, odec, owalk, G.TOL[cfg.dtype], G.MARGIN[cfg.dtype])
+    assert n == cfg.batch
+    assert np.array_equal(acc.numpy(), step.walk.accepted_node.cpu().numpy())
+    assert np.array_equal(hops.numpy(), step.walk.n_accepted.cpu().numpy())
+    assert np.array_equal(nxt.numpy(), step.walk.next_block.cpu().numpy())
+    assert int(step.decision.dev_status.max().item()) == 0
+    masked = int((w.block_tokens == cfg.mask_id).sum())
+    esz = host.logits.element_size()
+    assert step.h2d_bytes(host) == host.nbytes() - (host.logits.shape[:-1].numel() - masked) * cfg.vocab * esz
+    # unmasked rows were not copied
+    stale = torch.isnan(step.staging.logits.view(-1, cfg.vocab)[:, 0]).cpu().numpy()
+    assert np.array_equal(stale, (w.block_tokens != cfg.mask_id).reshape(-1))
