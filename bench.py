@@ -416,6 +416,7 @@ def main():
         t_attn = call_seconds(step.attention)
         t_dec = call_seconds(step.decide)
         t_walk = call_seconds(step.accept)
+        t_dw = call_seconds(step.decide_accept)
 
         # end to end from pinned host memory
         n_e2e = max(3, min(50, steps))
@@ -474,7 +475,7 @@ def main():
         "gpu_launches": int(round(launches_per_step * steps)),
         "roofline": roofline, "attention": attention,
         "per_call_us": {"graph_attention": t_attn * 1e6, "unmask_decide": t_dec * 1e6,
-                        "accept_walk": t_walk * 1e6},
+                        "accept_walk": t_walk * 1e6, "decide_walk": t_dw * 1e6},
         "dev_status": status,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -16,6 +16,8 @@
  *   spiffy_accept_walk       step 5 of Algorithm 1: the walk through the draft
  *                            graph (Sec. 4.4.1, Eqs. draft-graph-1..3) to the
  *                            deepest accepted node;
+ *   spiffy_decide_walk       the two above in one call (steps 1-5), fused on
+ *                            the device where the graph is small;
  *   spiffy_draft_blocks      drafting and pruning (Sec. 4.4.2, Sec. 4.4.4): the
  *                            draft blocks and parent lists of the next step.
  *
@@ -250,6 +252,26 @@ spiffy_status spiffy_accept_walk(const spiffy_decide_desc* desc,
                                  int32_t* accepted_node, int32_t* n_accepted,
                                  int32_t* path, int32_t* next_block,
                                  int32_t* dev_status, void* cuda_stream);
+
+/*
+ * Steps 1-5 of Algorithm 1 in one call: exactly spiffy_unmask_decide followed
+ * by spiffy_accept_walk on its top_tok / unmask_bits, with the same arguments,
+ * layouts, outputs (bit for bit) and status codes; decide_status and
+ * walk_status are the dev_status arrays of the two calls (either may be NULL).
+ * When a sequence's graph is small (N * L <= 512 and its arrays fit the
+ * default shared memory of one CTA) the merge of the vocabulary slices, the
+ * unmasking rule and the walk run in one kernel per sequence, one launch
+ * fewer than the two separate calls; otherwise this is the two calls.
+ * Workspace: spiffy_unmask_decide_workspace(desc).
+ */
+spiffy_status spiffy_decide_walk(const spiffy_decide_desc* desc, const void* logits,
+                                 const int32_t* block_tokens, const int32_t* parent_off,
+                                 const int32_t* parent_idx, int32_t parent_cap, float* conf,
+                                 int32_t* top_tok, uint64_t* unmask_bits, int32_t* n_unmask,
+                                 int32_t* decide_status, int32_t* accepted_node,
+                                 int32_t* n_accepted, int32_t* path, int32_t* next_block,
+                                 int32_t* walk_status, void* workspace, size_t workspace_bytes,
+                                 void* cuda_stream);
 
 /* ------------------------------------------------------------------------- */
 /* Drafting and pruning (Sec. 4.4.2 "Drafting Source", Sec. 4.4.4 "Pruning")  */

@@ -15,6 +15,7 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "walk_core.cuh"
 
 namespace spiffy {
 namespace {
@@ -53,7 +54,7 @@ __device__ __forceinline__ void merge(float& m, float& s, int& idx, float m2,
   const float M = fmaxf(m, m2);
   const float f1 = (m == M) ? 1.f : ex2((m - M) * kLog2e);
   const float f2 = (m2 == M) ? 1.f : ex2((m2 - M) * kLog2e);
-  s = s * f1 + s2 * f2;
+  s = __fmaf_rn(s, f1, __fmul_rn(s2, f2));  // spelled out: every instance rounds the same way
   m = M;
 }
 
@@ -146,9 +147,12 @@ __global__ void __launch_bounds__(kReduceThreads)
 decide_reduce_kernel(const T* __restrict__ logits, int64_t row_stride, int V,
                      int64_t chunk, int splits,
                      const int32_t* __restrict__ block_tokens, int mask_id,
-                     Partial* __restrict__ partials) {
+                     Partial* __restrict__ partials, int early_trigger) {
 #if __CUDA_ARCH__ >= 900
   cudaGridDependencySynchronize();  // inputs written by earlier kernels are visible
+  // The one-CTA-per-sequence tail kernel may take its SM while this grid still
+  // runs (it waits there for this grid to finish): its launch latency is hidden.
+  if (early_trigger) pdl_launch_dependents();
 #endif
   const int row = blockIdx.y;
   if (block_tokens[row] != mask_id) return;  // already unmasked: never read
@@ -225,8 +229,127 @@ decide_reduce_kernel(const T* __restrict__ logits, int64_t row_stride, int V,
   }
 }
 
+// kLanes (8, 4, 2 or 1) neighbouring lanes merge the slices of one row and lane
+// 0 of the group gets the row's confidence and top token (Algorithm 1, steps
+// 1-2).  The order is fixed and the same for every kLanes: eight accumulators
+// (accumulator j takes slices j, j + 8, ...) are combined by the butterfly
+// 4, 2, 1 with the lower index first; a lane holds the accumulators j = sub,
+// sub + kLanes, ... and does the butterfly steps that stay inside it locally.
+// Returns false on lane 0 when the row is masked and not usable.
+template <int kLanes>
+__device__ __forceinline__ bool finalize_row(const Partial* __restrict__ p, int splits, int sub,
+                                             int32_t state, int mask_id, float& conf, int32_t& tok) {
+  constexpr int kAcc = 8 / kLanes;
+  float m[kAcc], s[kAcc];
+  int idx[kAcc];
+#pragma unroll
+  for (int a = 0; a < kAcc; ++a) {
+    m[a] = -INFINITY;
+    s[a] = 0.f;
+    idx[a] = 0x7fffffff;
+  }
+  // this lane's slices are sub, sub + kLanes, sub + 2 kLanes, ...; slice number t
+  // goes to accumulator t mod kAcc.  They are fetched kBatch at a time, all
+  // loads of a batch in flight together; a missing slice merges as the identity.
+  constexpr int kBatch = kAcc > 4 ? kAcc : 4;
+  for (int t0 = 0; sub + kLanes * t0 < splits; t0 += kBatch) {
+    Partial q[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int k = sub + kLanes * (t0 + u);
+      q[u] = Partial{-INFINITY, 0.f, 0x7fffffff, 0};
+      if (k < splits) {  // read at L2: another grid wrote these while this CTA may already have been resident
+        const int4 w = __ldcg(reinterpret_cast<const int4*>(p + k));
+        q[u] = Partial{__int_as_float(w.x), __int_as_float(w.y), w.z, w.w};
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u)
+      merge(m[u % kAcc], s[u % kAcc], idx[u % kAcc], q[u].m, q[u].s, q[u].idx);
+  }
+#pragma unroll
+  for (int oa = kAcc / 2; oa > 0; oa >>= 1) {  // butterfly steps 4.. down to kLanes
+#pragma unroll
+    for (int a = 0; a < kAcc; ++a)
+      if (a < oa) merge(m[a], s[a], idx[a], m[a + oa], s[a + oa], idx[a + oa]);
+  }
+#pragma unroll
+  for (int off = kLanes / 2; off > 0; off >>= 1) {  // the remaining steps cross lanes
+    const float m2 = __shfl_xor_sync(0xffffffffu, m[0], off);
+    const float s2 = __shfl_xor_sync(0xffffffffu, s[0], off);
+    const int i2 = __shfl_xor_sync(0xffffffffu, idx[0], off);
+    merge(m[0], s[0], idx[0], m2, s2, i2);
+  }
+  const bool masked = state == mask_id;
+  conf = masked ? fminf(1.0f, 1.0f / s[0]) : -INFINITY;  // the sum can round just below one
+  tok = masked ? idx[0] : state;
+  // a usable row has a finite maximum and a finite, positive sum (the sum is one or more up to rounding)
+  return !(masked && (!(fabsf(m[0]) < INFINITY) || !(s[0] > 0.f) || !(s[0] < INFINITY)));
+}
+
+// One warp applies the unmasking rule of Sec. 3.1 (Algorithm 1, step 3) to one
+// node; lane k owns positions k and k + 32.  conf: the node's L confidences,
+// -inf at unmasked positions.  Returns the bit mask of positions to unmask.
+__device__ __forceinline__ uint64_t unmask_rule(const float* conf, const int32_t* state, int L,
+                                                int mask_id, int rule, int top_s, float tau,
+                                                int lane) {
+  const unsigned full = 0xffffffffu;
+  bool masked[2], take[2];
+  float c[2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int l = lane + 32 * h;
+    masked[h] = l < L && state[min(l, L - 1)] == mask_id;
+    c[h] = masked[h] ? conf[l] : -INFINITY;
+  }
+  if (rule == SPIFFY_RULE_TOPS && top_s > 1) {
+    // rank among the masked positions by (confidence desc, position asc); the
+    // confidence of an unmasked position is -inf and a masked one's is not
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int l = lane + 32 * h;
+      int rank = 0;
+      if (masked[h]) {
+        for (int j = 0; j < L; ++j) {
+          const float cj = conf[j];
+          rank += (cj > c[h] || (cj == c[h] && j < l)) ? 1 : 0;
+        }
+      }
+      take[h] = masked[h] && rank < top_s;
+    }
+  } else {
+    // only the single most confident masked position matters (top-1, or the
+    // fallback of the threshold rule): a warp arg-max, ties to the lower position
+    float bc = (c[0] == c[0]) ? c[0] : -INFINITY;  // an unusable row never wins
+    int bp = lane;
+    if (c[1] > bc) {
+      bc = c[1];
+      bp = lane + 32;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const float c2 = __shfl_xor_sync(full, bc, off);
+      const int p2 = __shfl_xor_sync(full, bp, off);
+      if (c2 > bc || (c2 == bc && p2 < bp)) {
+        bc = c2;
+        bp = p2;
+      }
+    }
+    const bool any_masked = __any_sync(full, masked[0] || masked[1]);
+    bool pass0 = false, pass1 = false;
+    if (rule != SPIFFY_RULE_TOPS) {
+      pass0 = masked[0] && c[0] > tau;  // strict, Sec. 3.1
+      pass1 = masked[1] && c[1] > tau;
+    }
+    const bool any_pass = __any_sync(full, pass0 || pass1);
+    take[0] = any_pass ? pass0 : (any_masked && masked[0] && bp == lane);
+    take[1] = any_pass ? pass1 : (any_masked && masked[1] && bp == lane + 32);
+  }
+  return (uint64_t)__ballot_sync(full, take[0]) | ((uint64_t)__ballot_sync(full, take[1]) << 32);
+}
+
 // grid = B*N nodes, 512 threads: eight threads per position merge the slices of
-// its row, then threads 0..63 apply the rule (thread l owns position l).
+// its row, then warp 0 applies the rule.
 constexpr int kFinalizeThreads = 512;
 __global__ void __launch_bounds__(kFinalizeThreads)
 decide_finalize_kernel(const Partial* __restrict__ partials, int splits, int N,
@@ -243,74 +366,120 @@ decide_finalize_kernel(const Partial* __restrict__ partials, int splits, int N,
   const int node = blockIdx.x;
   const int pos = threadIdx.x >> 3, sub = threadIdx.x & 7;
   __shared__ float sconf[64];
-  __shared__ uint32_t sballot[2];
-  if (threadIdx.x < 64) sconf[threadIdx.x] = -INFINITY;
-  __syncthreads();
   {
     const int row = node * L + min(pos, L - 1);
     // the token and the partials are read together (one trip to memory); the
-    // partials of an unmasked row were never written and are ignored below
+    // partials of an unmasked row were never written and are ignored
     const int32_t state = block_tokens[row];
-    float m = -INFINITY, s = 0.f;
-    int idx = 0x7fffffff;
-    const Partial* p = partials + (int64_t)row * splits;
-    for (int k = sub; k < splits; k += 8) {
-      const Partial q = p[k];
-      merge(m, s, idx, q.m, q.s, q.idx);
-    }
-#pragma unroll
-    for (int off = 4; off > 0; off >>= 1) {  // fixed order inside the group of eight
-      const float m2 = __shfl_xor_sync(0xffffffffu, m, off);
-      const float s2 = __shfl_xor_sync(0xffffffffu, s, off);
-      const int i2 = __shfl_xor_sync(0xffffffffu, idx, off);
-      merge(m, s, idx, m2, s2, i2);
-    }
+    float conf;
+    int32_t tok;
+    const bool ok = finalize_row<8>(partials + (int64_t)row * splits, splits, sub, state, mask_id, conf, tok);
     if (sub == 0 && pos < L) {
-      const bool masked = state == mask_id;
-      const float conf = masked ? fminf(1.0f, 1.0f / s) : -INFINITY;  // the sum can round just below one
       conf_out[row] = conf;
-      tok_out[row] = masked ? idx : state;
+      tok_out[row] = tok;
       sconf[pos] = conf;
-      // a usable row has a finite maximum and a finite, positive sum (the sum is one or more up to rounding)
-      if (masked && (!(fabsf(m) < INFINITY) || !(s > 0.f) || !(s < INFINITY))) {
-        if (dev_status) atomicOr(dev_status + node / N, SPIFFY_DEV_NONFINITE);
-      }
+      if (!ok && dev_status) atomicOr(dev_status + node / N, SPIFFY_DEV_NONFINITE);
     }
   }
   __syncthreads();
-  if (threadIdx.x >= 64) return;
-  const int l = threadIdx.x;
-  const bool masked = l < L && block_tokens[node * L + min(l, L - 1)] == mask_id;
-  const float conf = masked ? sconf[l] : -INFINITY;
-  // rank among the masked positions by (confidence desc, position asc); the
-  // confidence of an unmasked position is -inf and a masked one's is not
-  int rank = 0;
-  if (masked) {
-    for (int j = 0; j < L; ++j) {
-      const float c = sconf[j];
-      rank += (c > conf || (c == conf && j < l)) ? 1 : 0;
-    }
-  }
-  bool take;
-  if (rule == SPIFFY_RULE_TOPS) {
-    take = masked && rank < top_s;
-  } else {
-    const bool pass = masked && conf > tau;  // strict, Sec. 3.1
-    const uint32_t any0 = __ballot_sync(0xffffffffu, pass);
-    if ((l & 31) == 0) sballot[l >> 5] = any0;
-    asm volatile("bar.sync 1, 64;" ::: "memory");
-    const bool any = (sballot[0] | sballot[1]) != 0u;
-    asm volatile("bar.sync 1, 64;" ::: "memory");
-    take = any ? pass : (masked && rank == 0);
-  }
-  const uint32_t bal = __ballot_sync(0xffffffffu, take);
-  if ((l & 31) == 0) sballot[l >> 5] = bal;
-  asm volatile("bar.sync 1, 64;" ::: "memory");
-  if (l == 0) {
-    const uint64_t bits = (uint64_t)sballot[0] | ((uint64_t)sballot[1] << 32);
+  if (threadIdx.x >= 32) return;
+  const uint64_t bits = unmask_rule(sconf, block_tokens + (int64_t)node * L, L, mask_id, rule, top_s,
+                                    tau, threadIdx.x);
+  if (threadIdx.x == 0) {
     bits_out[node] = bits;
     n_unmask_out[node] = __popcll(bits);
   }
+}
+
+// Decision tail and acceptance walk of one sequence in one CTA (Algorithm 1,
+// steps 1-5 after the vocabulary reduce): eight threads per row merge the
+// slices, one warp per node applies the rule, warp 0 walks the draft graph with
+// every array it needs already in shared memory.  The graph (states, parent
+// lists) does not depend on the reduce kernel and is fetched before the wait on
+// it.  grid = B, kTailThreads threads, dynamic shared memory tail_smem_bytes().
+constexpr int kTailThreads = 1024;
+template <int kLanes>  // threads per row: all N * L rows are merged in one pass when kLanes * N * L <= 1024
+__global__ void __launch_bounds__(kTailThreads)
+decide_tail_kernel(const Partial* __restrict__ partials, int splits, int N, int L,
+                   const int32_t* __restrict__ block_tokens, int mask_id, int rule, int top_s,
+                   float tau, float* __restrict__ conf_out, int32_t* __restrict__ tok_out,
+                   uint64_t* __restrict__ bits_out, int32_t* __restrict__ n_unmask_out,
+                   int32_t* __restrict__ decide_status,
+                   const int32_t* __restrict__ parent_off, const int32_t* __restrict__ parent_idx,
+                   int parent_cap, int32_t* __restrict__ accepted_node,
+                   int32_t* __restrict__ n_accepted, int32_t* __restrict__ path,
+                   int32_t* __restrict__ next_block, int32_t* __restrict__ walk_status) {
+  extern __shared__ __align__(8) unsigned char tail_smem[];
+  const int b = blockIdx.x;
+  const int rows = N * L;
+  uint64_t* s_bits = reinterpret_cast<uint64_t*>(tail_smem);
+  int32_t* s_state = reinterpret_cast<int32_t*>(s_bits + N);
+  int32_t* s_top = s_state + rows;
+  float* s_conf = reinterpret_cast<float*>(s_top + rows);
+  int32_t* s_off = reinterpret_cast<int32_t*>(s_conf + rows);
+  int32_t* s_idx = s_off + (N + 1);
+  int* s_link = s_idx + parent_cap;
+  const int32_t* state = block_tokens + (int64_t)b * rows;
+  {
+    auto copy4 = [](void* dst, const void* src) {
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(
+                       (uint32_t)__cvta_generic_to_shared(dst)),
+                   "l"(src)
+                   : "memory");
+    };
+    const int32_t* off = parent_off + (int64_t)b * (N + 1);
+    const int32_t* idx = parent_idx + (int64_t)b * parent_cap;
+    for (int i = threadIdx.x; i < rows; i += kTailThreads) copy4(s_state + i, state + i);
+    for (int i = threadIdx.x; i <= N; i += kTailThreads) copy4(s_off + i, off + i);
+    for (int i = threadIdx.x; i < parent_cap; i += kTailThreads) copy4(s_idx + i, idx + i);
+    for (int i = threadIdx.x; i < N; i += kTailThreads) s_link[i] = kNoLink;
+  }
+#if __CUDA_ARCH__ >= 900
+  cudaGridDependencySynchronize();  // the reduce kernel's partials are visible
+  pdl_launch_dependents();          // only now: this CTA was resident during the reduce, the next kernel's need not be
+#endif
+  const int sub = threadIdx.x & (kLanes - 1);
+  for (int base = 0; base < rows; base += kTailThreads / kLanes) {
+    const int r = base + threadIdx.x / kLanes;
+    const int row = min(r, rows - 1);
+    const int32_t st = state[row];
+    float conf;
+    int32_t tok;
+    const bool ok = finalize_row<kLanes>(partials + ((int64_t)b * rows + row) * splits, splits, sub,
+                                         st, mask_id, conf, tok);
+    if (sub == 0 && r < rows) {
+      conf_out[(int64_t)b * rows + row] = conf;
+      tok_out[(int64_t)b * rows + row] = tok;
+      s_conf[row] = conf;
+      s_top[row] = tok;
+      if (!ok && decide_status) atomicOr(decide_status + b, SPIFFY_DEV_NONFINITE);
+    }
+  }
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int node = warp; node < N; node += kTailThreads / 32) {
+    const uint64_t bits = unmask_rule(s_conf + node * L, s_state + node * L, L, mask_id, rule, top_s,
+                                      tau, lane);
+    if (lane == 0) {
+      bits_out[(int64_t)b * N + node] = bits;
+      n_unmask_out[(int64_t)b * N + node] = __popcll(bits);
+      s_bits[node] = bits;
+    }
+  }
+  __syncthreads();
+  const bool bad = walk_link_children(N, L, parent_cap, s_state, s_top, s_off, s_idx, s_bits, s_link,
+                                      warp, kTailThreads / 32, lane);
+  if (bad && lane == 0 && walk_status) atomicOr(walk_status + b, SPIFFY_DEV_BADGRAPH);
+  __syncthreads();
+  if (warp == 0)
+    walk_chase(N, L, s_state, s_top, s_bits, s_link, path + (int64_t)b * N,
+               next_block + (int64_t)b * L, accepted_node + b, n_accepted + b, lane);
+}
+
+size_t tail_smem_bytes(const spiffy_decide_desc& d, int parent_cap) {
+  return (size_t)d.n_nodes * 8 +
+         ((size_t)3 * d.n_nodes * d.block_len + 2 * d.n_nodes + 1 + parent_cap) * 4;
 }
 
 }  // namespace
@@ -334,6 +503,28 @@ size_t decide_workspace_bytes(const spiffy_decide_desc& d) {
   return (size_t)rows * decide_splits(d, nullptr) * sizeof(Partial);
 }
 
+namespace {
+
+spiffy_status launch_reduce(const spiffy_decide_desc& d, const void* logits,
+                            const int32_t* block_tokens, Partial* partials, int splits,
+                            int64_t chunk, int early_trigger, cudaStream_t stream) {
+  const int rows = d.batch * d.n_nodes * d.block_len;
+  const dim3 grid(splits, rows);
+  cudaError_t e;
+  if (d.logits_dtype == SPIFFY_BF16)
+    e = launch_pdl(decide_reduce_kernel<__nv_bfloat16>, grid, dim3(kReduceThreads), (size_t)0, stream,
+                   static_cast<const __nv_bfloat16*>(logits), (int64_t)d.row_stride, (int)d.vocab,
+                   chunk, splits, block_tokens, (int)d.mask_token_id, partials, early_trigger);
+  else
+    e = launch_pdl(decide_reduce_kernel<float>, grid, dim3(kReduceThreads), (size_t)0, stream,
+                   static_cast<const float*>(logits), (int64_t)d.row_stride, (int)d.vocab, chunk,
+                   splits, block_tokens, (int)d.mask_token_id, partials, early_trigger);
+  count_launch();
+  return e == cudaSuccess ? SPIFFY_OK : SPIFFY_ECUDA;
+}
+
+}  // namespace
+
 spiffy_status launch_decide(const spiffy_decide_desc& d, const void* logits,
                             const int32_t* block_tokens, float* conf,
                             int32_t* top_tok, uint64_t* unmask_bits,
@@ -341,28 +532,59 @@ spiffy_status launch_decide(const spiffy_decide_desc& d, const void* logits,
                             cudaStream_t stream) {
   int64_t chunk = 0;
   const int splits = decide_splits(d, &chunk);
-  const int rows = d.batch * d.n_nodes * d.block_len;
   Partial* partials = static_cast<Partial*>(ws);
-  const dim3 grid(splits, rows);
-  cudaError_t e;
-  if (d.logits_dtype == SPIFFY_BF16)
-    e = launch_pdl(decide_reduce_kernel<__nv_bfloat16>, grid, dim3(kReduceThreads), (size_t)0, stream,
-                   static_cast<const __nv_bfloat16*>(logits), (int64_t)d.row_stride, (int)d.vocab,
-                   chunk, splits, block_tokens, (int)d.mask_token_id, partials);
-  else
-    e = launch_pdl(decide_reduce_kernel<float>, grid, dim3(kReduceThreads), (size_t)0, stream,
-                   static_cast<const float*>(logits), (int64_t)d.row_stride, (int)d.vocab, chunk,
-                   splits, block_tokens, (int)d.mask_token_id, partials);
-  count_launch();
-  if (e != cudaSuccess) return SPIFFY_ECUDA;
-
+  const spiffy_status st = launch_reduce(d, logits, block_tokens, partials, splits, chunk, 0, stream);
+  if (st != SPIFFY_OK) return st;
   // The finalize kernel's launch overlaps the tail of the reduce kernel; it
   // waits on the device (cudaGridDependencySynchronize) for the partials.
   const Partial* cpart = partials;
-  e = launch_pdl(decide_finalize_kernel, dim3(d.batch * d.n_nodes), dim3(kFinalizeThreads), (size_t)0, stream,
-                 cpart, splits, (int)d.n_nodes, (int)d.block_len, block_tokens,
+  const cudaError_t e =
+      launch_pdl(decide_finalize_kernel, dim3(d.batch * d.n_nodes), dim3(kFinalizeThreads), (size_t)0,
+                 stream, cpart, splits, (int)d.n_nodes, (int)d.block_len, block_tokens,
                  (int)d.mask_token_id, (int)d.rule, (int)d.top_s, d.threshold, conf, top_tok,
                  unmask_bits, n_unmask, dev_status);
+  count_launch();
+  return e == cudaSuccess ? SPIFFY_OK : SPIFFY_ECUDA;
+}
+
+// Decision and walk in one call.  Small graphs (at most kTailRows rows per
+// sequence, arrays within the default shared-memory limit) take the fused tail:
+// two launches instead of three.  Larger ones keep one finalize CTA per node,
+// which spreads the merging over more SMs.
+constexpr int kTailRows = 512;
+spiffy_status launch_decide_walk(const spiffy_decide_desc& d, const void* logits,
+                                 const int32_t* block_tokens, float* conf, int32_t* top_tok,
+                                 uint64_t* unmask_bits, int32_t* n_unmask,
+                                 int32_t* decide_status, const int32_t* parent_off,
+                                 const int32_t* parent_idx, int32_t parent_cap,
+                                 int32_t* accepted_node, int32_t* n_accepted, int32_t* path,
+                                 int32_t* next_block, int32_t* walk_status, void* ws,
+                                 cudaStream_t stream) {
+  const size_t smem = tail_smem_bytes(d, parent_cap);
+  if ((int64_t)d.n_nodes * d.block_len > kTailRows || smem > 48 * 1024) {
+    const spiffy_status st = launch_decide(d, logits, block_tokens, conf, top_tok, unmask_bits,
+                                           n_unmask, decide_status, ws, stream);
+    if (st != SPIFFY_OK) return st;
+    return launch_walk(d, block_tokens, parent_off, parent_idx, parent_cap, top_tok, unmask_bits,
+                       accepted_node, n_accepted, path, next_block, walk_status, stream);
+  }
+  int64_t chunk = 0;
+  const int splits = decide_splits(d, &chunk);
+  Partial* partials = static_cast<Partial*>(ws);
+  const spiffy_status st = launch_reduce(d, logits, block_tokens, partials, splits, chunk, 1, stream);
+  if (st != SPIFFY_OK) return st;
+  const Partial* cpart = partials;
+  const int rows = d.n_nodes * d.block_len;
+  auto launch = [&](auto kernel) {
+    return launch_pdl(kernel, dim3(d.batch), dim3(kTailThreads), smem, stream, cpart, splits,
+                      (int)d.n_nodes, (int)d.block_len, block_tokens, (int)d.mask_token_id,
+                      (int)d.rule, (int)d.top_s, d.threshold, conf, top_tok, unmask_bits, n_unmask,
+                      decide_status, parent_off, parent_idx, (int)parent_cap, accepted_node,
+                      n_accepted, path, next_block, walk_status);
+  };
+  const cudaError_t e = rows <= kTailThreads / 8   ? launch(decide_tail_kernel<8>)
+                        : rows <= kTailThreads / 4 ? launch(decide_tail_kernel<4>)
+                                                   : launch(decide_tail_kernel<2>);
   count_launch();
   return e == cudaSuccess ? SPIFFY_OK : SPIFFY_ECUDA;
 }

@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
         L.spiffy_draft_blocks.argtypes = [ctypes.POINTER(DraftDesc)] + [vp] * 14 + [sz, vp]
         L.spiffy_accept_walk.restype = ctypes.c_int
         L.spiffy_accept_walk.argtypes = [ctypes.POINTER(DecideDesc), vp, vp, vp, i32] + [vp] * 8
+        L.spiffy_decide_walk.restype = ctypes.c_int
+        L.spiffy_decide_walk.argtypes = [ctypes.POINTER(DecideDesc), vp, vp, vp, vp, i32] + [vp] * 11 + [sz, vp]
         L.spiffy_status_string.restype = ctypes.c_char_p
         L.spiffy_status_string.argtypes = [ctypes.c_int]
         L.spiffy_launch_count.restype = ctypes.c_uint64
@@ -281,6 +283,54 @@ def spiffy_accept_walk(block_tokens, parent_off, parent_idx, top_tok, unmask_bit
         _dev(out.dev_status, "dev_status", torch.int32), _stream(stream))
     _check(st, "spiffy_accept_walk")
     return out
+
+
+def _new_decision(B, N, L, dev) -> Decision:
+    return Decision(torch.empty((B, N, L), dtype=torch.float32, device=dev),
+                    torch.empty((B, N, L), dtype=torch.int32, device=dev),
+                    torch.empty((B, N), dtype=torch.int64, device=dev),
+                    torch.empty((B, N), dtype=torch.int32, device=dev),
+                    torch.zeros((B,), dtype=torch.int32, device=dev))
+
+
+def _new_walk(B, N, L, dev) -> Walk:
+    return Walk(torch.empty((B,), dtype=torch.int32, device=dev),
+                torch.empty((B,), dtype=torch.int32, device=dev),
+                torch.empty((B, N), dtype=torch.int32, device=dev),
+                torch.empty((B, L), dtype=torch.int32, device=dev),
+                torch.zeros((B,), dtype=torch.int32, device=dev))
+
+
+def spiffy_decide_walk(logits, block_tokens, parent_off, parent_idx, mask_token_id: int, rule: int,
+                       top_s: int = 1, threshold: float = 0.9, decision: Optional[Decision] = None,
+                       walk: Optional[Walk] = None, workspace=None, stream=None):
+    """Steps 1-5 of Algorithm 1 in one call: spiffy_unmask_decide followed by
+    spiffy_accept_walk, fused on the device for small graphs.  Returns
+    (Decision, Walk)."""
+    desc = decide_desc(logits, block_tokens, mask_token_id, rule, top_s, threshold)
+    B, N, L = block_tokens.shape
+    dev = logits.device
+    decision = decision or _new_decision(B, N, L, dev)
+    walk = walk or _new_walk(B, N, L, dev)
+    if tuple(parent_off.shape) != (B, N + 1) or parent_idx.dim() != 2 or parent_idx.shape[0] != B:
+        raise ValueError("parent_off must be [B,N+1] and parent_idx [B,cap]")
+    if workspace is None:
+        workspace = torch.empty(max(spiffy_unmask_decide_workspace(desc), 16), dtype=torch.uint8, device=dev)
+    st = lib().spiffy_decide_walk(
+        ctypes.byref(desc), _logits_ptr(logits), _dev(block_tokens, "block_tokens", torch.int32),
+        _dev(parent_off, "parent_off", torch.int32), _dev(parent_idx, "parent_idx", torch.int32),
+        int(parent_idx.shape[1]),
+        _dev(decision.conf, "conf", torch.float32), _dev(decision.top_tok, "top_tok", torch.int32),
+        _dev(decision.unmask_bits, "unmask_bits", torch.int64),
+        _dev(decision.n_unmask, "n_unmask", torch.int32),
+        _dev(decision.dev_status, "decide_status", torch.int32),
+        _dev(walk.accepted_node, "accepted_node", torch.int32),
+        _dev(walk.n_accepted, "n_accepted", torch.int32), _dev(walk.path, "path", torch.int32),
+        _dev(walk.next_block, "next_block", torch.int32),
+        _dev(walk.dev_status, "walk_status", torch.int32), _dev(workspace, "workspace"),
+        workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(st, "spiffy_decide_walk")
+    return decision, walk
 
 
 @dataclass

@@ -124,10 +124,16 @@ class VerifyStep:
                                          self.decision.top_tok, self.decision.unmask_bits,
                                          out=self.walk)
 
+    def decide_accept(self, x: StepInputs):
+        c = self.cfg
+        spiffy.spiffy_decide_walk(x.logits, x.block_tokens, x.parent_off, x.parent_idx, c.mask_id,
+                                  c.rule, c.top_s, c.threshold, decision=self.decision,
+                                  walk=self.walk, workspace=self.decide_ws)
+        return self.walk
+
     def run(self, x: StepInputs):
         self.attention(x)
-        self.decide(x)
-        return self.accept(x)
+        return self.decide_accept(x)
 
     @staticmethod
     def _masked_row_runs(host: StepInputs, mask_id: int):

@@ -50,8 +50,22 @@ def gpu_decide(w, logits_dev=None):
     dec = spiffy.spiffy_unmask_decide(logits, tokens, cfg.mask_id, cfg.rule, cfg.top_s, cfg.threshold)
     walk = spiffy.spiffy_accept_walk(tokens, to_dev(w.parent_off), to_dev(w.parent_idx),
                                      dec.top_tok, dec.unmask_bits)
+    # the one-call form gives the same bits, whichever kernels it takes
+    dec2, walk2 = spiffy.spiffy_decide_walk(logits, tokens, to_dev(w.parent_off), to_dev(w.parent_idx),
+                                            cfg.mask_id, cfg.rule, cfg.top_s, cfg.threshold)
     torch.cuda.synchronize()
+    assert_same_bits(dec, walk, dec2, walk2)
     return dec, walk
+
+
+def assert_same_bits(dec, walk, dec2, walk2):
+    """Two runs of the decision and the walk agree bit for bit (confidences are
+    compared as integers so that a NaN equals itself)."""
+    assert torch.equal(dec.conf.view(torch.int32), dec2.conf.view(torch.int32))
+    for f in ("top_tok", "unmask_bits", "n_unmask", "dev_status"):
+        assert torch.equal(getattr(dec, f), getattr(dec2, f)), f
+    for f in ("accepted_node", "n_accepted", "path", "next_block", "dev_status"):
+        assert torch.equal(getattr(walk, f), getattr(walk2, f)), f
 
 
 def oracle_decide(w):
