@@ -97,6 +97,29 @@ def test_walk_rejects_bad_arguments(lib):
     assert lib.spiffy_accept_walk(ctypes.byref(d), *neg) == spiffy.EINVAL
 
 
+def test_decide_walk_rejects_bad_arguments(lib):
+    """The one-call form checks what the two calls check, before any launch."""
+    fake = ctypes.c_void_p(0x1000)
+
+    def call(d, logits=fake, parent_off=fake, cap=4, next_block=fake, ws=fake, ws_bytes=1 << 30):
+        # desc, logits, tokens, parent_off, parent_idx, cap, conf, top_tok, bits, n_unmask, decide_status,
+        # accepted_node, n_accepted, path, next_block, walk_status, workspace, bytes, stream
+        return lib.spiffy_decide_walk(ctypes.byref(d), logits, fake, parent_off, fake, cap, fake, fake, fake,
+                                      fake, None, fake, fake, fake, next_block, None, ws, ws_bytes, None)
+
+    good = spiffy.DecideDesc(1, 2, 4, 32, spiffy.F32, 32, 31, spiffy.RULE_TOPS, 1, 0.0)
+    assert call(good, logits=None) == spiffy.EINVAL
+    assert call(good, parent_off=None) == spiffy.EINVAL
+    assert call(good, next_block=None) == spiffy.EINVAL
+    assert call(good, cap=-1) == spiffy.EINVAL
+    assert call(good, logits=ctypes.c_void_p(0x1004)) == spiffy.EINVAL
+    assert call(good, ws=None) == spiffy.EWORKSPACE
+    assert call(good, ws_bytes=8) == spiffy.EWORKSPACE
+    assert call(spiffy.DecideDesc(1, 2, 65, 32, spiffy.F32, 32, 31, spiffy.RULE_TOPS, 1, 0.0)) == spiffy.EUNSUPPORTED
+    assert call(spiffy.DecideDesc(1, 2, 4, 32, spiffy.F32, 32, 31, 7, 1, 0.0)) == spiffy.EINVAL
+    assert call(spiffy.DecideDesc(1, 2, 4, 33, spiffy.F32, 33, 31, spiffy.RULE_TOPS, 1, 0.0)) == spiffy.EINVAL
+
+
 def test_draft_rejects_bad_arguments(lib):
     fake = ctypes.c_void_p(0x1000)
 
