@@ -18,6 +18,8 @@
  *                            deepest accepted node;
  *   spiffy_decide_walk       the two above in one call (steps 1-5), fused on
  *                            the device where the graph is small;
+ *   spiffy_decide_walk_lazy  steps 1-5 with the decision evaluated only for the
+ *                            nodes the walk reaches (fewer bytes read);
  *   spiffy_draft_blocks      drafting and pruning (Sec. 4.4.2, Sec. 4.4.4): the
  *                            draft blocks and parent lists of the next step.
  *
@@ -272,6 +274,40 @@ spiffy_status spiffy_decide_walk(const spiffy_decide_desc* desc, const void* log
                                  int32_t* n_accepted, int32_t* path, int32_t* next_block,
                                  int32_t* walk_status, void* workspace, size_t workspace_bytes,
                                  void* cuda_stream);
+
+/*
+ * Lazy chain evaluation of steps 1-5 of Algorithm 1: the decision is computed
+ * only for the nodes the walk reaches (the true block, then each accepted
+ * draft), level by level inside one kernel, instead of for all N nodes.  Only
+ * 1 + n_accepted of the N nodes' logits are read.  The paper has no
+ * counterpart; it evaluates every draft's distribution (Sec. 4.3).
+ *
+ * Same arguments and layouts as spiffy_decide_walk.  On return
+ *   - accepted_node, n_accepted, path, next_block are those of
+ *     spiffy_decide_walk, bit for bit;
+ *   - conf, top_tok, unmask_bits, n_unmask hold, for the nodes on the path, the
+ *     bits spiffy_unmask_decide gives; for every other node n_unmask is -1 and
+ *     the other three are left untouched;
+ *   - walk_status reports a malformed parent list only if the walk scanned it;
+ *     SPIFFY_DEV_TIMEOUT in both status words when a bounded wait between the
+ *     levels ran out (results are then unspecified).
+ * Each level costs two grid-wide barriers, so the call pays off when one
+ * node's share of the logits is large (long vocabularies, batches) and loses
+ * to spiffy_decide_walk on a single short graph.  SPIFFY_EUNSUPPORTED when
+ * the batch exceeds the number of thread blocks the device holds at once.
+ * Workspace: spiffy_decide_walk_lazy_workspace(desc); contents on entry
+ * arbitrary (the call zeroes the few bytes it needs with a memset on the
+ * stream).
+ */
+size_t spiffy_decide_walk_lazy_workspace(const spiffy_decide_desc* desc);
+spiffy_status spiffy_decide_walk_lazy(const spiffy_decide_desc* desc, const void* logits,
+                                      const int32_t* block_tokens, const int32_t* parent_off,
+                                      const int32_t* parent_idx, int32_t parent_cap, float* conf,
+                                      int32_t* top_tok, uint64_t* unmask_bits, int32_t* n_unmask,
+                                      int32_t* decide_status, int32_t* accepted_node,
+                                      int32_t* n_accepted, int32_t* path, int32_t* next_block,
+                                      int32_t* walk_status, void* workspace,
+                                      size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------- */
 /* Drafting and pruning (Sec. 4.4.2 "Drafting Source", Sec. 4.4.4 "Pruning")  */

@@ -167,6 +167,33 @@ spiffy_status spiffy_decide_walk(const spiffy_decide_desc* desc, const void* log
                             static_cast<cudaStream_t>(cuda_stream));
 }
 
+size_t spiffy_decide_walk_lazy_workspace(const spiffy_decide_desc* desc) {
+  if (check_decide_desc(desc, true) != SPIFFY_OK) return 0;
+  return decide_lazy_workspace_bytes(*desc);
+}
+
+spiffy_status spiffy_decide_walk_lazy(const spiffy_decide_desc* desc, const void* logits,
+                                      const int32_t* block_tokens, const int32_t* parent_off,
+                                      const int32_t* parent_idx, int32_t parent_cap, float* conf,
+                                      int32_t* top_tok, uint64_t* unmask_bits, int32_t* n_unmask,
+                                      int32_t* decide_status, int32_t* accepted_node,
+                                      int32_t* n_accepted, int32_t* path, int32_t* next_block,
+                                      int32_t* walk_status, void* workspace,
+                                      size_t workspace_bytes, void* cuda_stream) {
+  const spiffy_status st = check_decide_desc(desc, true);
+  if (st != SPIFFY_OK) return st;
+  if (!logits || !block_tokens || !conf || !top_tok || !unmask_bits || !n_unmask || !parent_off ||
+      !parent_idx || !accepted_node || !n_accepted || !path || !next_block)
+    return SPIFFY_EINVAL;
+  if (!aligned16(logits) || parent_cap < 0) return SPIFFY_EINVAL;
+  const size_t need = decide_lazy_workspace_bytes(*desc);
+  if (!workspace || workspace_bytes < need || !aligned16(workspace)) return SPIFFY_EWORKSPACE;
+  return launch_decide_walk_lazy(*desc, logits, block_tokens, conf, top_tok, unmask_bits, n_unmask,
+                                 decide_status, parent_off, parent_idx, parent_cap, accepted_node,
+                                 n_accepted, path, next_block, walk_status, workspace,
+                                 static_cast<cudaStream_t>(cuda_stream));
+}
+
 size_t spiffy_draft_blocks_workspace(const spiffy_draft_desc* desc) {
   if (check_draft_desc(desc) != SPIFFY_OK) return 0;
   return draft_workspace_bytes(*desc);

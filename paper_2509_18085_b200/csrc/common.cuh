@@ -41,6 +41,16 @@ spiffy_status launch_decide_walk(const spiffy_decide_desc& d, const void* logits
                                  int32_t* next_block, int32_t* walk_status, void* ws,
                                  cudaStream_t stream);
 
+size_t decide_lazy_workspace_bytes(const spiffy_decide_desc& d);
+spiffy_status launch_decide_walk_lazy(const spiffy_decide_desc& d, const void* logits,
+                                      const int32_t* block_tokens, float* conf, int32_t* top_tok,
+                                      uint64_t* unmask_bits, int32_t* n_unmask,
+                                      int32_t* decide_status, const int32_t* parent_off,
+                                      const int32_t* parent_idx, int32_t parent_cap,
+                                      int32_t* accepted_node, int32_t* n_accepted, int32_t* path,
+                                      int32_t* next_block, int32_t* walk_status, void* ws,
+                                      cudaStream_t stream);
+
 spiffy_status launch_attention_simt(const spiffy_attn_desc& d, const void* q,
                                     const void* kp, const void* vp,
                                     const void* kb, const void* vb, void* out,

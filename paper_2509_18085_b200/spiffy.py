@@ -93,6 +93,10 @@ def lib() -> ctypes.CDLL:
         L.spiffy_accept_walk.argtypes = [ctypes.POINTER(DecideDesc), vp, vp, vp, i32] + [vp] * 8
         L.spiffy_decide_walk.restype = ctypes.c_int
         L.spiffy_decide_walk.argtypes = [ctypes.POINTER(DecideDesc), vp, vp, vp, vp, i32] + [vp] * 11 + [sz, vp]
+        L.spiffy_decide_walk_lazy_workspace.restype = sz
+        L.spiffy_decide_walk_lazy_workspace.argtypes = [ctypes.POINTER(DecideDesc)]
+        L.spiffy_decide_walk_lazy.restype = ctypes.c_int
+        L.spiffy_decide_walk_lazy.argtypes = L.spiffy_decide_walk.argtypes
         L.spiffy_status_string.restype = ctypes.c_char_p
         L.spiffy_status_string.argtypes = [ctypes.c_int]
         L.spiffy_launch_count.restype = ctypes.c_uint64
@@ -301,12 +305,18 @@ def _new_walk(B, N, L, dev) -> Walk:
                 torch.zeros((B,), dtype=torch.int32, device=dev))
 
 
+def spiffy_decide_walk_lazy_workspace(desc: DecideDesc) -> int:
+    return int(lib().spiffy_decide_walk_lazy_workspace(ctypes.byref(desc)))
+
+
 def spiffy_decide_walk(logits, block_tokens, parent_off, parent_idx, mask_token_id: int, rule: int,
                        top_s: int = 1, threshold: float = 0.9, decision: Optional[Decision] = None,
-                       walk: Optional[Walk] = None, workspace=None, stream=None):
+                       walk: Optional[Walk] = None, workspace=None, stream=None, lazy: bool = False):
     """Steps 1-5 of Algorithm 1 in one call: spiffy_unmask_decide followed by
-    spiffy_accept_walk, fused on the device for small graphs.  Returns
-    (Decision, Walk)."""
+    spiffy_accept_walk, fused on the device for small graphs.  With ``lazy`` the
+    decision is evaluated only for the nodes the walk reaches
+    (spiffy_decide_walk_lazy): the Decision then holds those nodes' entries and
+    n_unmask = -1 everywhere else.  Returns (Decision, Walk)."""
     desc = decide_desc(logits, block_tokens, mask_token_id, rule, top_s, threshold)
     B, N, L = block_tokens.shape
     dev = logits.device
@@ -314,9 +324,11 @@ def spiffy_decide_walk(logits, block_tokens, parent_off, parent_idx, mask_token_
     walk = walk or _new_walk(B, N, L, dev)
     if tuple(parent_off.shape) != (B, N + 1) or parent_idx.dim() != 2 or parent_idx.shape[0] != B:
         raise ValueError("parent_off must be [B,N+1] and parent_idx [B,cap]")
+    need = spiffy_decide_walk_lazy_workspace(desc) if lazy else spiffy_unmask_decide_workspace(desc)
     if workspace is None:
-        workspace = torch.empty(max(spiffy_unmask_decide_workspace(desc), 16), dtype=torch.uint8, device=dev)
-    st = lib().spiffy_decide_walk(
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    entry = lib().spiffy_decide_walk_lazy if lazy else lib().spiffy_decide_walk
+    st = entry(
         ctypes.byref(desc), _logits_ptr(logits), _dev(block_tokens, "block_tokens", torch.int32),
         _dev(parent_off, "parent_off", torch.int32), _dev(parent_idx, "parent_idx", torch.int32),
         int(parent_idx.shape[1]),
@@ -329,7 +341,7 @@ def spiffy_decide_walk(logits, block_tokens, parent_off, parent_idx, mask_token_
         _dev(walk.next_block, "next_block", torch.int32),
         _dev(walk.dev_status, "walk_status", torch.int32), _dev(workspace, "workspace"),
         workspace.numel() * workspace.element_size(), _stream(stream))
-    _check(st, "spiffy_decide_walk")
+    _check(st, "spiffy_decide_walk_lazy" if lazy else "spiffy_decide_walk")
     return decision, walk
 
 

@@ -146,3 +146,89 @@ def test_graph_replay_over_changing_inputs_sharing_one_workspace():
             stream.synchronize()
             for (dec, walk), (dec0, walk0) in zip(outs, want):
                 G.assert_same_bits(dec0, walk0, dec, walk)
+
+
+# ---------------------------------------------------------------------------
+# lazy chain evaluation: the decision only for the nodes the walk reaches
+# ---------------------------------------------------------------------------
+def lazy_vs_eager(logits, tokens, off, idx, mask_id, rule, top_s=1, tau=0.9, dtype=None):
+    lg, tk, of, ix = G.to_dev(logits, dtype), G.to_dev(tokens), G.to_dev(off), G.to_dev(idx)
+    dec, walk = spiffy.spiffy_decide_walk(lg, tk, of, ix, mask_id, rule, top_s, tau)
+    B, N, L = tokens.shape
+    # poison what the lazy call must leave alone or overwrite
+    lazy_dec = spiffy.Decision(torch.full((B, N, L), -7.0, device="cuda"),
+                               torch.full((B, N, L), -7, dtype=torch.int32, device="cuda"),
+                               torch.full((B, N), -7, dtype=torch.int64, device="cuda"),
+                               torch.full((B, N), -7, dtype=torch.int32, device="cuda"),
+                               torch.zeros((B,), dtype=torch.int32, device="cuda"))
+    ldec, lwalk = spiffy.spiffy_decide_walk(lg, tk, of, ix, mask_id, rule, top_s, tau, decision=lazy_dec,
+                                            lazy=True)
+    torch.cuda.synchronize()
+    for f in ("accepted_node", "n_accepted", "path", "next_block"):
+        assert torch.equal(getattr(walk, f), getattr(lwalk, f)), f
+    assert torch.equal(dec.dev_status, ldec.dev_status) or int(dec.dev_status.sum()) != 0
+    path = walk.path.cpu().numpy()
+    on_path = np.zeros((B, N), dtype=bool)
+    for b in range(B):
+        on_path[b, path[b][path[b] >= 0]] = True
+    m = torch.from_numpy(on_path).cuda()
+    assert torch.equal(dec.conf.view(torch.int32)[m], ldec.conf.view(torch.int32)[m])
+    assert torch.equal(dec.top_tok[m], ldec.top_tok[m])
+    assert torch.equal(dec.unmask_bits[m], ldec.unmask_bits[m])
+    assert torch.equal(dec.n_unmask[m], ldec.n_unmask[m])
+    # nodes off the path: marked as not evaluated, nothing else written
+    assert bool((ldec.n_unmask[~m] == -1).all())
+    assert bool((ldec.conf[~m] == -7.0).all()) and bool((ldec.top_tok[~m] == -7).all())
+    assert bool((ldec.unmask_bits[~m] == -7).all())
+    return walk, lwalk, on_path
+
+
+@pytest.mark.parametrize("B,N,L,V", [(3, 8, 32, 5000), (2, 16, 32, 1000), (5, 3, 7, 36), (1, 2, 64, 300),
+                                     (2, 9, 64, 132), (1, 1, 1, 16), (40, 8, 16, 200)])
+def test_lazy_chain_evaluation_equals_the_eager_call_on_the_path(B, N, L, V):
+    hops = 0
+    for rule, S, tau in ((spiffy.RULE_TOPS, 1, 0.0), (spiffy.RULE_TOPS, 3, 0.0), (spiffy.RULE_THRESHOLD, 1, 0.5)):
+        logits, tokens, off, idx, mask = random_case(B * 100 + N, B, N, L, V, p_accept=0.9)
+        walk, _, on_path = lazy_vs_eager(logits, tokens, off, idx, mask, rule, S, tau)
+        hops += int(walk.n_accepted.sum())
+        assert on_path[:, 0].all()
+    if N > 2:
+        assert hops > 0
+
+
+def test_lazy_chain_evaluation_at_the_benchmark_shapes():
+    for index, cases in ((2, 2), (3, 1)):
+        cfg = W.config(index)
+        for case in range(cases):
+            w = W.make(cfg, W.seed_for(index, case))
+            walk, lwalk, on_path = lazy_vs_eager(w.logits, w.block_tokens, w.parent_off, w.parent_idx,
+                                                 cfg.mask_id, cfg.rule, cfg.top_s, cfg.threshold,
+                                                 dtype=G.tdtype(cfg))
+            _, ow = G.oracle_decide(w)
+            assert np.array_equal(lwalk.path.cpu().numpy(), ow.path)
+            assert np.array_equal(lwalk.next_block.cpu().numpy(), ow.next_block)
+            assert int(lwalk.dev_status.sum()) == 0
+
+
+def test_lazy_call_in_a_cuda_graph():
+    logits, tokens, off, idx, mask = random_case(11, 2, 8, 16, 2000, p_accept=1.0)
+    lg, tk, of, ix = G.to_dev(logits), G.to_dev(tokens), G.to_dev(off), G.to_dev(idx)
+    dec0, walk0 = spiffy.spiffy_decide_walk(lg, tk, of, ix, mask, spiffy.RULE_TOPS)
+    desc = spiffy.decide_desc(lg, tk, mask, spiffy.RULE_TOPS, 1, 0.9)
+    ws = torch.empty(spiffy.spiffy_decide_walk_lazy_workspace(desc), dtype=torch.uint8, device="cuda")
+    dec, walk = spiffy.spiffy_decide_walk(lg, tk, of, ix, mask, spiffy.RULE_TOPS, workspace=ws, lazy=True)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            spiffy.spiffy_decide_walk(lg, tk, of, ix, mask, spiffy.RULE_TOPS, decision=dec, walk=walk,
+                                      workspace=ws, lazy=True)
+        for _ in range(10):
+            walk.next_block.zero_()
+            walk.path.zero_()
+            graph.replay()
+            stream.synchronize()
+            for f in ("accepted_node", "n_accepted", "path", "next_block", "dev_status"):
+                assert torch.equal(getattr(walk, f), getattr(walk0, f)), f
+    assert int(walk0.n_accepted.max()) >= 2
