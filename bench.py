@@ -56,7 +56,7 @@ def parse():
     ap.add_argument("--nodes", type=int, default=None, help="node count for configuration 5")
     ap.add_argument("--attn-kernel", default="auto", choices=["auto", "simt", "tcgen05"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--part", default="step", choices=["step", "attention", "decide", "draft"],
+    ap.add_argument("--part", default="step", choices=["step", "attention", "decide", "decide_walk", "decide_walk_lazy", "draft"],
                     help="time one library call alone on any configuration (for profiling); "
                          "the benchmark line itself is --part step")
     ap.add_argument("--sets", type=int, default=0, help="rotating input sets for --part (0 = enough to exceed L2)")
@@ -244,7 +244,8 @@ def run_part(args):
     sets = [inputs_from_workload(w) for w in work]
     kernel = {"auto": spiffy.ATTN_AUTO, "simt": spiffy.ATTN_SIMT, "tcgen05": spiffy.ATTN_TCGEN05}[args.attn_kernel]
     step = VerifyStep(cfg, attn_kernel=kernel)
-    call = step.attention if attn else step.decide
+    call = {"attention": step.attention, "decide": step.decide, "decide_walk": step.decide_accept,
+            "decide_walk_lazy": step.decide_accept_lazy}[args.part]
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
         for x in sets:
@@ -277,6 +278,20 @@ def run_part(args):
         by = algorithmic_bytes(cfg, masked_all)[1]
         out.update(gbs=by / sec / 1e9, frac_of_hbm=by / sec / 1e9 / peaks["hbm_gbs"], algorithmic_bytes=by,
                    masked_rows=masked_all)
+        if args.part == "decide_walk_lazy":
+            # what the lazy call has to read: the still-masked rows of the nodes on the accepted path
+            rows, hops = [], []
+            for x, w in zip(sets, work):
+                walk = call(x)
+                torch.cuda.synchronize()
+                path = walk.path.cpu().numpy()
+                hops.append(float(walk.n_accepted.float().mean()))
+                rows.append(sum(int((w.block_tokens[b, n] == cfg.mask_id).sum())
+                                for b in range(cfg.batch) for n in path[b] if n >= 0))
+            lazy_by = algorithmic_bytes(cfg, float(np.mean(rows)))[1]
+            out.update(rows_on_path=float(np.mean(rows)), mean_accepted=float(np.mean(hops)),
+                       lazy_algorithmic_bytes=lazy_by, lazy_gbs=lazy_by / sec / 1e9,
+                       note="gbs counts the eager call's bytes (every node); lazy_gbs the bytes this call reads")
     out["peaks"] = peaks["source"]
     print(json.dumps(out))
 

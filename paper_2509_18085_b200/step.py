@@ -107,6 +107,7 @@ class VerifyStep:
         self.verdict_host = (host(self.walk.accepted_node), host(self.walk.n_accepted),
                              host(self.walk.next_block))
         self.staging = None
+        self.lazy_ws = None
 
     # the three calls of one step, asynchronous on the current stream
     def attention(self, x: StepInputs):
@@ -129,6 +130,18 @@ class VerifyStep:
         spiffy.spiffy_decide_walk(x.logits, x.block_tokens, x.parent_off, x.parent_idx, c.mask_id,
                                   c.rule, c.top_s, c.threshold, decision=self.decision,
                                   walk=self.walk, workspace=self.decide_ws)
+        return self.walk
+
+    def decide_accept_lazy(self, x: StepInputs):
+        """The decision only for the nodes the walk reaches (spiffy_decide_walk_lazy)."""
+        c = self.cfg
+        if self.lazy_ws is None:
+            desc = spiffy.decide_desc(x.logits, x.block_tokens, c.mask_id, c.rule, c.top_s, c.threshold)
+            self.lazy_ws = torch.empty((max(16, spiffy.spiffy_decide_walk_lazy_workspace(desc)),),
+                                       dtype=torch.uint8, device=self.device)
+        spiffy.spiffy_decide_walk(x.logits, x.block_tokens, x.parent_off, x.parent_idx, c.mask_id,
+                                  c.rule, c.top_s, c.threshold, decision=self.decision,
+                                  walk=self.walk, workspace=self.lazy_ws, lazy=True)
         return self.walk
 
     def run(self, x: StepInputs):
