@@ -120,6 +120,28 @@ def test_decide_walk_rejects_bad_arguments(lib):
     assert call(spiffy.DecideDesc(1, 2, 4, 33, spiffy.F32, 33, 31, spiffy.RULE_TOPS, 1, 0.0)) == spiffy.EINVAL
 
 
+def test_lazy_decide_walk_rejects_bad_arguments(lib):
+    fake = ctypes.c_void_p(0x1000)
+    good = spiffy.DecideDesc(2, 4, 8, 1024, spiffy.BF16, 1024, 1023, spiffy.RULE_THRESHOLD, 1, 0.9)
+    need = lib.spiffy_decide_walk_lazy_workspace(ctypes.byref(good))
+    # partial results of one node per sequence, plus the header and three words per sequence
+    assert need >= 2 * 8 * 16 + 16 + 2 * 12
+    assert need < lib.spiffy_unmask_decide_workspace(ctypes.byref(good)) + 64
+
+    def call(d, logits=fake, parent_idx=fake, cap=4, ws=fake, ws_bytes=1 << 30):
+        return lib.spiffy_decide_walk_lazy(ctypes.byref(d), logits, fake, fake, parent_idx, cap, fake, fake,
+                                           fake, fake, None, fake, fake, fake, fake, None, ws, ws_bytes, None)
+
+    assert call(good, logits=None) == spiffy.EINVAL
+    assert call(good, parent_idx=None) == spiffy.EINVAL
+    assert call(good, cap=-2) == spiffy.EINVAL
+    assert call(good, ws=None) == spiffy.EWORKSPACE
+    assert call(good, ws_bytes=need - 1) == spiffy.EWORKSPACE
+    bad = spiffy.DecideDesc(2, 4, 8, 1024, spiffy.BF16, 1024, 1023, spiffy.RULE_TOPS, 0, 0.9)
+    assert call(bad) == spiffy.EINVAL
+    assert lib.spiffy_decide_walk_lazy_workspace(ctypes.byref(bad)) == 0
+
+
 def test_draft_rejects_bad_arguments(lib):
     fake = ctypes.c_void_p(0x1000)
 
