@@ -309,6 +309,23 @@ spiffy_status spiffy_decide_walk_lazy(const spiffy_decide_desc* desc, const void
                                       int32_t* walk_status, void* workspace,
                                       size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * Staging helper for callers whose logits sit in pinned host memory (the paper
+ * has no counterpart: its logits never leave the device).  Copies row r
+ * (row_bytes bytes, a multiple of 16) from src_rows to dst_rows for every r in
+ * [0, n_rows) with tokens[r] == mask_token_id, i.e. exactly the rows
+ * spiffy_unmask_decide will read; other rows of dst_rows are left as they are.
+ *   src_rows, tokens: memory the DEVICE can read -- device memory, or pinned
+ *             host memory that is mapped into the device's address space (with
+ *             unified addressing every cudaHostAlloc / cudaHostRegister
+ *             allocation is); 16-byte aligned
+ *   dst_rows: device memory, 16-byte aligned, same row layout as src_rows
+ * One kernel reads the rows over the bus; n_rows <= 65535.
+ */
+spiffy_status spiffy_stage_masked_rows(const void* src_rows, void* dst_rows, int64_t row_bytes,
+                                       const int32_t* tokens, int32_t mask_token_id,
+                                       int64_t n_rows, void* cuda_stream);
+
 /* ------------------------------------------------------------------------- */
 /* Drafting and pruning (Sec. 4.4.2 "Drafting Source", Sec. 4.4.4 "Pruning")  */
 /* ------------------------------------------------------------------------- */

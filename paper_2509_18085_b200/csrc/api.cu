@@ -194,6 +194,17 @@ spiffy_status spiffy_decide_walk_lazy(const spiffy_decide_desc* desc, const void
                                  static_cast<cudaStream_t>(cuda_stream));
 }
 
+spiffy_status spiffy_stage_masked_rows(const void* src_rows, void* dst_rows, int64_t row_bytes,
+                                       const int32_t* tokens, int32_t mask_token_id,
+                                       int64_t n_rows, void* cuda_stream) {
+  if (!src_rows || !dst_rows || !tokens) return SPIFFY_EINVAL;
+  if (row_bytes < 16 || row_bytes % 16 != 0 || n_rows < 1) return SPIFFY_EINVAL;
+  if (!aligned16(src_rows) || !aligned16(dst_rows)) return SPIFFY_EINVAL;
+  if (n_rows > 65535) return SPIFFY_EUNSUPPORTED;
+  return launch_stage_masked_rows(src_rows, dst_rows, row_bytes, tokens, mask_token_id, n_rows,
+                                  static_cast<cudaStream_t>(cuda_stream));
+}
+
 size_t spiffy_draft_blocks_workspace(const spiffy_draft_desc* desc) {
   if (check_draft_desc(desc) != SPIFFY_OK) return 0;
   return draft_workspace_bytes(*desc);

@@ -51,6 +51,10 @@ spiffy_status launch_decide_walk_lazy(const spiffy_decide_desc& d, const void* l
                                       int32_t* next_block, int32_t* walk_status, void* ws,
                                       cudaStream_t stream);
 
+spiffy_status launch_stage_masked_rows(const void* src, void* dst, int64_t row_bytes,
+                                       const int32_t* tokens, int32_t mask_id, int64_t n_rows,
+                                       cudaStream_t stream);
+
 spiffy_status launch_attention_simt(const spiffy_attn_desc& d, const void* q,
                                     const void* kp, const void* vp,
                                     const void* kb, const void* vb, void* out,

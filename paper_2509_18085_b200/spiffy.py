@@ -97,6 +97,8 @@ def lib() -> ctypes.CDLL:
         L.spiffy_decide_walk_lazy_workspace.argtypes = [ctypes.POINTER(DecideDesc)]
         L.spiffy_decide_walk_lazy.restype = ctypes.c_int
         L.spiffy_decide_walk_lazy.argtypes = L.spiffy_decide_walk.argtypes
+        L.spiffy_stage_masked_rows.restype = ctypes.c_int
+        L.spiffy_stage_masked_rows.argtypes = [vp, vp, ctypes.c_int64, vp, i32, ctypes.c_int64, vp]
         L.spiffy_status_string.restype = ctypes.c_char_p
         L.spiffy_status_string.argtypes = [ctypes.c_int]
         L.spiffy_launch_count.restype = ctypes.c_uint64
@@ -343,6 +345,29 @@ def spiffy_decide_walk(logits, block_tokens, parent_off, parent_idx, mask_token_
         workspace.numel() * workspace.element_size(), _stream(stream))
     _check(st, "spiffy_decide_walk_lazy" if lazy else "spiffy_decide_walk")
     return decision, walk
+
+
+def spiffy_stage_masked_rows(src_logits, dst_logits, tokens, mask_token_id: int, stream=None):
+    """Copies the logits rows of still-masked positions from ``src_logits`` (a
+    pinned host tensor, or a device tensor) into the device tensor
+    ``dst_logits`` of the same shape; ``tokens`` (pinned host or device int32)
+    has one entry per row."""
+    if not dst_logits.is_cuda or not dst_logits.is_contiguous():
+        raise ValueError("dst_logits must be a contiguous CUDA tensor")
+    for name, t in (("src_logits", src_logits), ("tokens", tokens)):
+        if not (t.is_cuda or t.is_pinned()) or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous CUDA or pinned host tensor")
+    if src_logits.shape != dst_logits.shape or src_logits.dtype != dst_logits.dtype:
+        raise ValueError("src_logits and dst_logits differ in shape or dtype")
+    if tokens.dtype != torch.int32 or tokens.numel() != src_logits.numel() // src_logits.shape[-1]:
+        raise ValueError("tokens must be int32 with one entry per logits row")
+    row_bytes = src_logits.shape[-1] * src_logits.element_size()
+    st = lib().spiffy_stage_masked_rows(ctypes.c_void_p(src_logits.data_ptr()),
+                                        ctypes.c_void_p(dst_logits.data_ptr()), row_bytes,
+                                        ctypes.c_void_p(tokens.data_ptr()), int(mask_token_id),
+                                        tokens.numel(), _stream(stream))
+    _check(st, "spiffy_stage_masked_rows")
+    return dst_logits
 
 
 @dataclass

@@ -9,7 +9,6 @@ and copies the verdict back -- the end-to-end call.
 """
 from __future__ import annotations
 
-import ctypes
 from dataclasses import dataclass
 
 import torch
@@ -55,22 +54,6 @@ def inputs_from_workload(w, device="cuda", pin=False) -> StepInputs:
                       mv(w.parent_idx))
 
 
-_CUDART = None
-
-
-def _cudart():
-    """The CUDA runtime torch has loaded, for row-run copies without a tensor
-    slice per run."""
-    global _CUDART
-    if _CUDART is None:
-        major = torch.version.cuda.split(".")[0]
-        _CUDART = ctypes.CDLL(f"libcudart.so.{major}")
-        _CUDART.cudaMemcpyAsync.restype = ctypes.c_int
-        _CUDART.cudaMemcpyAsync.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int,
-                                            ctypes.c_void_p]
-    return _CUDART
-
-
 class VerifyStep:
     def __init__(self, cfg: Config, device="cuda", attn_kernel=spiffy.ATTN_AUTO):
         self.cfg = cfg
@@ -108,6 +91,8 @@ class VerifyStep:
                              host(self.walk.next_block))
         self.staging = None
         self.lazy_ws = None
+        self.copy_stream = None
+        self.copy_events = None
 
     # the three calls of one step, asynchronous on the current stream
     def attention(self, x: StepInputs):
@@ -159,23 +144,27 @@ class VerifyStep:
     def run_host(self, host: StepInputs):
         """End to end from pinned host memory: copy the step's inputs in, run
         it, read the verdict (accepted node, hop count, next block) back.  Of
-        the logits only the rows of still-masked positions cross the bus (runs
-        of neighbouring rows in one copy each); the staging rows of unmasked
-        positions keep whatever they held and no kernel reads them."""
+        the logits only the rows of still-masked positions cross the bus
+        (spiffy_stage_masked_rows reads them from the pinned buffer); the
+        staging rows of unmasked positions keep whatever they held and no
+        kernel reads them."""
         if self.staging is None:
             self.staging = StepInputs(*[torch.empty_like(t, device=self.device) for t in host.tensors()])
-        row = host.logits.shape[-1] * host.logits.element_size()
-        base_dst, base_src = self.staging.logits.data_ptr(), host.logits.data_ptr()
-        stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
-        copy = _cudart().cudaMemcpyAsync
-        for a, b in self._masked_row_runs(host, self.cfg.mask_id):
-            rc = copy(ctypes.c_void_p(base_dst + a * row), ctypes.c_void_p(base_src + a * row),
-                      ctypes.c_size_t((b - a) * row), 1, stream)  # 1 = host to device
-            if rc != 0:
-                raise RuntimeError(f"cudaMemcpyAsync failed with error {rc}")
-        for dst, src in zip(self.staging.tensors(), host.tensors()):
-            if src is not host.logits:
-                dst.copy_(src, non_blocking=True)
+        main = torch.cuda.current_stream()
+        if self.copy_stream is None:
+            self.copy_stream = torch.cuda.Stream(self.device)
+            self.copy_events = (torch.cuda.Event(), torch.cuda.Event())
+        # the small tensors go through the copy engine on a side stream while one kernel pulls
+        # the masked logits rows over the bus; both start once the staging buffers are free
+        self.copy_events[0].record(main)
+        self.copy_stream.wait_event(self.copy_events[0])
+        with torch.cuda.stream(self.copy_stream):
+            for dst, src in zip(self.staging.tensors(), host.tensors()):
+                if src is not host.logits:
+                    dst.copy_(src, non_blocking=True)
+            self.copy_events[1].record(self.copy_stream)
+        spiffy.spiffy_stage_masked_rows(host.logits, self.staging.logits, host.block_tokens, self.cfg.mask_id)
+        main.wait_event(self.copy_events[1])
         w = self.run(self.staging)
         for dst, src in zip(self.verdict_host, (w.accepted_node, w.n_accepted, w.next_block)):
             dst.copy_(src, non_blocking=True)

@@ -142,6 +142,20 @@ def test_lazy_decide_walk_rejects_bad_arguments(lib):
     assert lib.spiffy_decide_walk_lazy_workspace(ctypes.byref(bad)) == 0
 
 
+def test_stage_masked_rows_rejects_bad_arguments(lib):
+    fake = ctypes.c_void_p(0x1000)
+    call = lambda src=fake, dst=fake, row_bytes=256, tokens=fake, rows=4: lib.spiffy_stage_masked_rows(
+        src, dst, row_bytes, tokens, 7, rows, None)
+    assert call(src=None) == spiffy.EINVAL
+    assert call(dst=None) == spiffy.EINVAL
+    assert call(tokens=None) == spiffy.EINVAL
+    assert call(row_bytes=0) == spiffy.EINVAL
+    assert call(row_bytes=250) == spiffy.EINVAL            # rows must be whole 16-byte vectors
+    assert call(src=ctypes.c_void_p(0x1008)) == spiffy.EINVAL
+    assert call(rows=0) == spiffy.EINVAL
+    assert call(rows=70000) == spiffy.EUNSUPPORTED
+
+
 def test_draft_rejects_bad_arguments(lib):
     fake = ctypes.c_void_p(0x1000)
 

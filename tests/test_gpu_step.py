@@ -228,3 +228,29 @@ def test_end_to_end_call_from_host_memory(config):
     # unmasked rows were not copied
     stale = torch.isnan(step.staging.logits.view(-1, cfg.vocab)[:, 0]).cpu().numpy()
     assert np.array_equal(stale, (w.block_tokens != cfg.mask_id).reshape(-1))
+
+
+@pytest.mark.parametrize("dtype,V", [(torch.bfloat16, 126464), (torch.float32, 1000), (torch.bfloat16, 8),
+                                     (torch.float32, 2052)])
+@pytest.mark.parametrize("pinned", [True, False])
+def test_stage_masked_rows_copies_exactly_the_masked_rows(dtype, V, pinned):
+    """From pinned host memory or device memory: masked rows arrive bit for
+    bit, every other row of the destination keeps what it held."""
+    rows = 37
+    g = torch.Generator().manual_seed(V)
+    src = torch.randn((rows, V), generator=g).to(dtype)
+    tokens = torch.where(torch.rand(rows, generator=g) < 0.6, 9, 3).to(torch.int32)
+    tokens[0], tokens[-1] = 9, 3
+    if pinned:
+        src_in, tok_in = src.pin_memory(), tokens.pin_memory()
+    else:
+        src_in, tok_in = src.cuda(), tokens.cuda()
+    dst = torch.full((rows, V), 5.0, dtype=dtype, device="cuda")
+    spiffy.spiffy_stage_masked_rows(src_in, dst, tok_in, 9)
+    torch.cuda.synchronize()
+    got = dst.cpu()
+    masked = tokens == 9
+    assert torch.equal(got[masked].view(torch.uint8), src[masked].view(torch.uint8))
+    assert bool((got[~masked] == 5.0).all())
+    with pytest.raises(ValueError):
+        spiffy.spiffy_stage_masked_rows(src, dst, tok_in, 9)  # pageable host memory
