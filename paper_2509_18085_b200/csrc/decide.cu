@@ -21,7 +21,7 @@ namespace {
 
 // grid = (splits, B*N*L); one CTA reduces one vocabulary slice of one row.
 template <typename T>
-__global__ void __launch_bounds__(kReduceThreads)
+__global__ void __launch_bounds__(kReduceThreads, 8)  // 64 registers: eight CTAs per SM
 decide_reduce_kernel(const T* __restrict__ logits, int64_t row_stride, int V,
                      int64_t chunk, int splits,
                      const int32_t* __restrict__ block_tokens, int mask_id,

@@ -35,6 +35,34 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// Two fp32 lanes in one 64-bit register: Blackwell issues their multiply-add and
+// their add as one instruction each (the kernel is bound by instruction issue).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+// acc += {2^(x0 * log2e - ml), 2^(x1 * log2e - ml)}; k2 = {log2e, log2e}, nml2 = {-ml, -ml}
+__device__ __forceinline__ uint64_t add_exp2(uint64_t acc, float x0, float x1, uint64_t k2,
+                                             uint64_t nml2) {
+  float a0, a1;
+  unpack2(fma2(pack2(x0, x1), k2, nml2), a0, a1);
+  return add2(acc, pack2(ex2(a0), ex2(a1)));
+}
+
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   uint4 v;
   asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -71,6 +99,12 @@ struct Elem<__nv_bfloat16> {
     const __nv_bfloat162 p = __hmax2(__hmax2(pk(v.x), pk(v.y)), __hmax2(pk(v.z), pk(v.w)));
     return fmaxf(__low2float(p), __high2float(p));
   }
+  // true when some element of the vector equals x (x is one of the inputs, hence a bf16 value)
+  static __device__ __forceinline__ bool holds(uint4 v, float x) {
+    const __nv_bfloat162 xx = __float2bfloat162_rn(x);
+    return (__heq2_mask(pk(v.x), xx) | __heq2_mask(pk(v.y), xx) | __heq2_mask(pk(v.z), xx) |
+            __heq2_mask(pk(v.w), xx)) != 0u;
+  }
   static __device__ __forceinline__ float gmax(const uint4 (&v)[kUnroll]) {
     __nv_bfloat162 p = __hmax2(__hmax2(pk(v[0].x), pk(v[0].y)), __hmax2(pk(v[0].z), pk(v[0].w)));
 #pragma unroll
@@ -78,14 +112,14 @@ struct Elem<__nv_bfloat16> {
       p = __hmax2(p, __hmax2(__hmax2(pk(v[k].x), pk(v[k].y)), __hmax2(pk(v[k].z), pk(v[k].w))));
     return fmaxf(__low2float(p), __high2float(p));
   }
-  // sum over the vector of 2^(x * log2e - ml)
-  static __device__ __forceinline__ float sum_terms(uint4 v, float ml) {
+  // acc (two running sums) += 2^(x * log2e - ml) over the vector, even elements into the
+  // low lane, odd ones into the high lane
+  static __device__ __forceinline__ uint64_t sum_terms(uint4 v, uint64_t k2, uint64_t nml2,
+                                                       uint64_t acc) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    float t = 0.f;
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
-      t += ex2(fmaf(lo(w[i]), kLog2e, -ml)) + ex2(fmaf(hi(w[i]), kLog2e, -ml));
-    return t;
+    for (int i = 0; i < 4; ++i) acc = add_exp2(acc, lo(w[i]), hi(w[i]), k2, nml2);
+    return acc;
   }
   // position of the first element equal to x, kPerVec if there is none
   static __device__ __forceinline__ int first_equal(uint4 v, float x) {
@@ -111,6 +145,7 @@ struct Elem<float> {
     return fmaxf(fmaxf(__uint_as_float(v.x), __uint_as_float(v.y)),
                  fmaxf(__uint_as_float(v.z), __uint_as_float(v.w)));
   }
+  static __device__ __forceinline__ bool holds(uint4 v, float x) { return vmax(v) == x; }
   static __device__ __forceinline__ float gmax(const uint4 (&v)[kUnroll]) {
     float g = -INFINITY;
 #pragma unroll
@@ -119,9 +154,10 @@ struct Elem<float> {
                          fmaxf(__uint_as_float(v[k].z), __uint_as_float(v[k].w))));
     return g;
   }
-  static __device__ __forceinline__ float sum_terms(uint4 v, float ml) {
-    return (ex2(fmaf(__uint_as_float(v.x), kLog2e, -ml)) + ex2(fmaf(__uint_as_float(v.y), kLog2e, -ml))) +
-           (ex2(fmaf(__uint_as_float(v.z), kLog2e, -ml)) + ex2(fmaf(__uint_as_float(v.w), kLog2e, -ml)));
+  static __device__ __forceinline__ uint64_t sum_terms(uint4 v, uint64_t k2, uint64_t nml2,
+                                                       uint64_t acc) {
+    acc = add_exp2(acc, __uint_as_float(v.x), __uint_as_float(v.y), k2, nml2);
+    return add_exp2(acc, __uint_as_float(v.z), __uint_as_float(v.w), k2, nml2);
   }
   static __device__ __forceinline__ int first_equal(uint4 v, float x) {
     int j = kPerVec;
@@ -179,13 +215,20 @@ __device__ __forceinline__ void reduce_slice(const T* __restrict__ base, int V, 
   for (int w = 1; w < kReduceThreads / 32; ++w) m = fmaxf(m, warp_m[w]);
   // 3. sum of exp(x - m) and the lowest index that attains m
   const float ml = (m == -INFINITY) ? 0.f : m * kLog2e;  // an all -inf slice sums to 0
-  float s = 0.f;
+  const uint64_t k2 = pack2(kLog2e, kLog2e), nml2 = pack2(-ml, -ml);
+  uint64_t acc = pack2(0.f, 0.f);
   int idx = 0x7fffffff;
 #pragma unroll
   for (int u = kUnroll - 1; u >= 0; --u) {
-    s += Elem<T>::sum_terms(v[u], ml);
-    if (Elem<T>::vmax(v[u]) == m)  // rare: only the vectors that hold the slice maximum are searched
+    acc = Elem<T>::sum_terms(v[u], k2, nml2, acc);
+    if (Elem<T>::holds(v[u], m))  // rare: only the vectors that hold the slice maximum are searched
       idx = (int)begin + (tid + u * kReduceThreads) * EPV + Elem<T>::first_equal(v[u], m);
+  }
+  float s;
+  {
+    float s0, s1;
+    unpack2(acc, s0, s1);
+    s = s0 + s1;
   }
   if (ntail > 0 && tid == 0) {
     int tidx = 0x7fffffff;
