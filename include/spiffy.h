@@ -21,7 +21,11 @@
  *   spiffy_decide_walk_lazy  steps 1-5 with the decision evaluated only for the
  *                            nodes the walk reaches (fewer bytes read);
  *   spiffy_draft_blocks      drafting and pruning (Sec. 4.4.2, Sec. 4.4.4): the
- *                            draft blocks and parent lists of the next step.
+ *                            draft blocks and parent lists of the next step;
+ *   spiffy_stage_masked_rows, spiffy_unmask_decide_static
+ *                            helpers without a counterpart in the paper: staging
+ *                            of logits from pinned host memory, and the decision
+ *                            step with its scratch inside the library.
  *
  * Vocabulary (paper notation in brackets where it differs):
  *   B  batch of independent sequences            N  nodes of the draft graph,
@@ -32,8 +36,9 @@
  *   tau  confidence threshold of dynamic unmasking; S  static unmasking rate
  *
  * Conventions common to every entry point
- *   - Every data pointer is a DEVICE pointer owned by the caller; the library
- *     neither allocates nor frees device memory.  Descriptors are plain host
+ *   - Every data pointer is a DEVICE pointer owned by the caller (the source of
+ *     spiffy_stage_masked_rows may also be mapped pinned host memory); the
+ *     library neither allocates nor frees device memory.  Descriptors are plain host
  *     structs, read before the call returns.
  *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*,
  *     NULL = the default stream) and never synchronise the device.
