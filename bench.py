@@ -56,7 +56,7 @@ def parse():
     ap.add_argument("--nodes", type=int, default=None, help="node count for configuration 5")
     ap.add_argument("--attn-kernel", default="auto", choices=["auto", "simt", "tcgen05"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--part", default="step", choices=["step", "attention", "decide", "decide_walk", "decide_walk_lazy", "draft"],
+    ap.add_argument("--part", default="step", choices=["step", "attention", "decide", "decide_walk", "decide_walk_lazy", "decide_sampled", "draft"],
                     help="time one library call alone on any configuration (for profiling); "
                          "the benchmark line itself is --part step")
     ap.add_argument("--sets", type=int, default=0, help="rotating input sets for --part (0 = enough to exceed L2)")
@@ -245,7 +245,7 @@ def run_part(args):
     kernel = {"auto": spiffy.ATTN_AUTO, "simt": spiffy.ATTN_SIMT, "tcgen05": spiffy.ATTN_TCGEN05}[args.attn_kernel]
     step = VerifyStep(cfg, attn_kernel=kernel)
     call = {"attention": step.attention, "decide": step.decide, "decide_walk": step.decide_accept,
-            "decide_walk_lazy": step.decide_accept_lazy}[args.part]
+            "decide_walk_lazy": step.decide_accept_lazy, "decide_sampled": step.decide_sampled}[args.part]
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
         for x in sets:

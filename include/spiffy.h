@@ -20,6 +20,8 @@
  *                            the device where the graph is small;
  *   spiffy_decide_walk_lazy  steps 1-5 with the decision evaluated only for the
  *                            nodes the walk reaches (fewer bytes read);
+ *   spiffy_unmask_decide_sampled
+ *                            steps 1-4 at sampling temperature T > 0;
  *   spiffy_draft_blocks      drafting and pruning (Sec. 4.4.2, Sec. 4.4.4): the
  *                            draft blocks and parent lists of the next step;
  *   spiffy_stage_masked_rows, spiffy_unmask_decide_static
@@ -223,6 +225,40 @@ spiffy_status spiffy_unmask_decide_static(const spiffy_decide_desc* desc,
                                           int32_t* n_unmask,
                                           int32_t* dev_status,
                                           void* cuda_stream);
+
+/*
+ * The decision step at sampling temperature T > 0 (Sec. 5.4 runs Spiffy at
+ * T > 0; the sampler itself is not given in the paper and is fixed here).
+ * Per still-masked position the token is drawn from softmax(x / T) as
+ *   top_tok = argmax_v (x_v / T + g_v),  g_v = -ln(-ln u_v)      (Gumbel-max)
+ * and conf is its probability softmax(x / T)[top_tok]; the unmasking rule then
+ * runs on conf exactly as in spiffy_unmask_decide, and every other argument,
+ * layout and status bit is that call's.
+ * The uniforms u_v come from the counter-based generator Philox4x32-10
+ * (Salmon, Moraes, Dror, Shaw, SC 2011):
+ *   counter = (v / 4, position l, sequence b, number of still-masked positions
+ *              of the node),  key = (seed & 0xffffffff, seed >> 32),
+ *   u_v = (output word v % 4 + 0.5) / 2^32.
+ * The noise depends on the state of the block, not on the node's index: a
+ * draft block and the true block that equals it draw the same tokens, which is
+ * what the losslessness argument of App. A needs.  A caller that wants fresh
+ * noise for another block or request changes the seed.
+ * Workspace: spiffy_unmask_decide_sampled_workspace(desc).
+ */
+typedef struct {
+  float temperature; /* T > 0 */
+  uint32_t reserved; /* 0 */
+  uint64_t seed;
+} spiffy_sample_desc;
+
+size_t spiffy_unmask_decide_sampled_workspace(const spiffy_decide_desc* desc);
+spiffy_status spiffy_unmask_decide_sampled(const spiffy_decide_desc* desc,
+                                           const spiffy_sample_desc* sample, const void* logits,
+                                           const int32_t* block_tokens, float* conf,
+                                           int32_t* top_tok, uint64_t* unmask_bits,
+                                           int32_t* n_unmask, int32_t* dev_status,
+                                           void* workspace, size_t workspace_bytes,
+                                           void* cuda_stream);
 
 /* ------------------------------------------------------------------------- */
 /* Acceptance: step 5 of Algorithm 1 over the draft graph of Sec. 4.4.1      */

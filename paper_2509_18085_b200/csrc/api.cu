@@ -205,6 +205,31 @@ spiffy_status spiffy_stage_masked_rows(const void* src_rows, void* dst_rows, int
                                   static_cast<cudaStream_t>(cuda_stream));
 }
 
+size_t spiffy_unmask_decide_sampled_workspace(const spiffy_decide_desc* desc) {
+  if (check_decide_desc(desc, true) != SPIFFY_OK) return 0;
+  return decide_sampled_workspace_bytes(*desc);
+}
+
+spiffy_status spiffy_unmask_decide_sampled(const spiffy_decide_desc* desc,
+                                           const spiffy_sample_desc* sample, const void* logits,
+                                           const int32_t* block_tokens, float* conf,
+                                           int32_t* top_tok, uint64_t* unmask_bits,
+                                           int32_t* n_unmask, int32_t* dev_status,
+                                           void* workspace, size_t workspace_bytes,
+                                           void* cuda_stream) {
+  const spiffy_status st = check_decide_desc(desc, true);
+  if (st != SPIFFY_OK) return st;
+  if (!sample || !(sample->temperature > 0.f) || !(sample->temperature < INFINITY)) return SPIFFY_EINVAL;
+  if (!logits || !block_tokens || !conf || !top_tok || !unmask_bits || !n_unmask)
+    return SPIFFY_EINVAL;
+  if (!aligned16(logits)) return SPIFFY_EINVAL;
+  const size_t need = decide_sampled_workspace_bytes(*desc);
+  if (!workspace || workspace_bytes < need || !aligned16(workspace)) return SPIFFY_EWORKSPACE;
+  return launch_decide_sampled(*desc, sample->temperature, sample->seed, logits, block_tokens, conf,
+                               top_tok, unmask_bits, n_unmask, dev_status, workspace,
+                               static_cast<cudaStream_t>(cuda_stream));
+}
+
 size_t spiffy_draft_blocks_workspace(const spiffy_draft_desc* desc) {
   if (check_draft_desc(desc) != SPIFFY_OK) return 0;
   return draft_workspace_bytes(*desc);

@@ -55,6 +55,12 @@ spiffy_status launch_stage_masked_rows(const void* src, void* dst, int64_t row_b
                                        const int32_t* tokens, int32_t mask_id, int64_t n_rows,
                                        cudaStream_t stream);
 
+size_t decide_sampled_workspace_bytes(const spiffy_decide_desc& d);
+spiffy_status launch_decide_sampled(const spiffy_decide_desc& d, float temperature, uint64_t seed,
+                                    const void* logits, const int32_t* block_tokens, float* conf,
+                                    int32_t* top_tok, uint64_t* unmask_bits, int32_t* n_unmask,
+                                    int32_t* dev_status, void* ws, cudaStream_t stream);
+
 spiffy_status launch_attention_simt(const spiffy_attn_desc& d, const void* q,
                                     const void* kp, const void* vp,
                                     const void* kb, const void* vb, void* out,

@@ -55,6 +55,10 @@ class DecideDesc(ctypes.Structure):
                 ("top_s", ctypes.c_int32), ("threshold", ctypes.c_float)]
 
 
+class SampleDesc(ctypes.Structure):
+    _fields_ = [("temperature", ctypes.c_float), ("reserved", ctypes.c_uint32), ("seed", ctypes.c_uint64)]
+
+
 class DraftDesc(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("block_len", ctypes.c_int32), ("vocab", ctypes.c_int32),
                 ("logits_dtype", ctypes.c_int32), ("row_stride", ctypes.c_int64),
@@ -99,6 +103,11 @@ def lib() -> ctypes.CDLL:
         L.spiffy_decide_walk_lazy.argtypes = L.spiffy_decide_walk.argtypes
         L.spiffy_stage_masked_rows.restype = ctypes.c_int
         L.spiffy_stage_masked_rows.argtypes = [vp, vp, ctypes.c_int64, vp, i32, ctypes.c_int64, vp]
+        L.spiffy_unmask_decide_sampled_workspace.restype = sz
+        L.spiffy_unmask_decide_sampled_workspace.argtypes = [ctypes.POINTER(DecideDesc)]
+        L.spiffy_unmask_decide_sampled.restype = ctypes.c_int
+        L.spiffy_unmask_decide_sampled.argtypes = [ctypes.POINTER(DecideDesc), ctypes.POINTER(SampleDesc)] + \
+            [vp] * 8 + [sz, vp]
         L.spiffy_status_string.restype = ctypes.c_char_p
         L.spiffy_status_string.argtypes = [ctypes.c_int]
         L.spiffy_launch_count.restype = ctypes.c_uint64
@@ -233,6 +242,38 @@ def spiffy_unmask_decide(logits, block_tokens, mask_token_id: int, rule: int,
         _dev(out.dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
         workspace.numel() * workspace.element_size(), _stream(stream))
     _check(st, "spiffy_unmask_decide")
+    return out
+
+
+def spiffy_unmask_decide_sampled(logits, block_tokens, mask_token_id: int, rule: int, temperature: float,
+                                 seed: int, top_s: int = 1, threshold: float = 0.9,
+                                 out: Optional[Decision] = None, workspace=None, stream=None) -> Decision:
+    """Steps 1-4 of Algorithm 1 at sampling temperature T > 0: tokens drawn from
+    softmax(x / T) by Gumbel-max with Philox4x32-10 noise that follows the
+    block's state (sequence, position, vocabulary entry, masked count), never
+    the node's index; conf is the drawn token's probability."""
+    desc = decide_desc(logits, block_tokens, mask_token_id, rule, top_s, threshold)
+    sample = SampleDesc(float(temperature), 0, int(seed) & 0xFFFFFFFFFFFFFFFF)
+    B, N, L = block_tokens.shape
+    dev = logits.device
+    if out is None:
+        out = Decision(torch.empty((B, N, L), dtype=torch.float32, device=dev),
+                       torch.empty((B, N, L), dtype=torch.int32, device=dev),
+                       torch.empty((B, N), dtype=torch.int64, device=dev),
+                       torch.empty((B, N), dtype=torch.int32, device=dev),
+                       torch.zeros((B,), dtype=torch.int32, device=dev))
+    if workspace is None:
+        need = int(lib().spiffy_unmask_decide_sampled_workspace(ctypes.byref(desc)))
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    st = lib().spiffy_unmask_decide_sampled(
+        ctypes.byref(desc), ctypes.byref(sample), _logits_ptr(logits),
+        _dev(block_tokens, "block_tokens", torch.int32),
+        _dev(out.conf, "conf", torch.float32), _dev(out.top_tok, "top_tok", torch.int32),
+        _dev(out.unmask_bits, "unmask_bits", torch.int64),
+        _dev(out.n_unmask, "n_unmask", torch.int32),
+        _dev(out.dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
+        workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(st, "spiffy_unmask_decide_sampled")
     return out
 
 

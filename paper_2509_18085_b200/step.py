@@ -9,6 +9,7 @@ and copies the verdict back -- the end-to-end call.
 """
 from __future__ import annotations
 
+import ctypes
 from dataclasses import dataclass
 
 import torch
@@ -91,6 +92,7 @@ class VerifyStep:
                              host(self.walk.next_block))
         self.staging = None
         self.lazy_ws = None
+        self.sampled_ws = None
         self.copy_stream = None
         self.copy_events = None
 
@@ -116,6 +118,17 @@ class VerifyStep:
                                   c.rule, c.top_s, c.threshold, decision=self.decision,
                                   walk=self.walk, workspace=self.decide_ws)
         return self.walk
+
+    def decide_sampled(self, x: StepInputs, temperature: float = 1.0, seed: int = 1):
+        """The decision at sampling temperature T > 0 (spiffy_unmask_decide_sampled)."""
+        c = self.cfg
+        if self.sampled_ws is None:
+            desc = spiffy.decide_desc(x.logits, x.block_tokens, c.mask_id, c.rule, c.top_s, c.threshold)
+            need = int(spiffy.lib().spiffy_unmask_decide_sampled_workspace(ctypes.byref(desc)))
+            self.sampled_ws = torch.empty((max(16, need),), dtype=torch.uint8, device=self.device)
+        return spiffy.spiffy_unmask_decide_sampled(x.logits, x.block_tokens, c.mask_id, c.rule, temperature,
+                                                   seed, c.top_s, c.threshold, out=self.decision,
+                                                   workspace=self.sampled_ws)
 
     def decide_accept_lazy(self, x: StepInputs):
         """The decision only for the nodes the walk reaches (spiffy_decide_walk_lazy)."""

@@ -156,6 +156,27 @@ def test_stage_masked_rows_rejects_bad_arguments(lib):
     assert call(rows=70000) == spiffy.EUNSUPPORTED
 
 
+def test_sampled_decide_rejects_bad_arguments(lib):
+    fake = ctypes.c_void_p(0x1000)
+    good = spiffy.DecideDesc(1, 4, 8, 1024, spiffy.BF16, 1024, 1023, spiffy.RULE_TOPS, 1, 0.9)
+    need = lib.spiffy_unmask_decide_sampled_workspace(ctypes.byref(good))
+    assert need == 2 * lib.spiffy_unmask_decide_workspace(ctypes.byref(good))  # 32-byte partial results
+
+    def call(temperature=1.0, sample=True, logits=fake, ws=fake, ws_bytes=1 << 30, d=good):
+        s = spiffy.SampleDesc(temperature, 0, 42)
+        return lib.spiffy_unmask_decide_sampled(ctypes.byref(d), ctypes.byref(s) if sample else None, logits,
+                                                fake, fake, fake, fake, fake, None, ws, ws_bytes, None)
+
+    assert call(sample=False) == spiffy.EINVAL
+    for t in (0.0, -0.5, float("nan"), float("inf")):
+        assert call(temperature=t) == spiffy.EINVAL
+    assert call(logits=None) == spiffy.EINVAL
+    assert call(ws=None) == spiffy.EWORKSPACE
+    assert call(ws_bytes=need - 1) == spiffy.EWORKSPACE
+    assert call(d=spiffy.DecideDesc(1, 4, 65, 1024, spiffy.BF16, 1024, 1023, spiffy.RULE_TOPS, 1, 0.9)) == \
+        spiffy.EUNSUPPORTED
+
+
 def test_draft_rejects_bad_arguments(lib):
     fake = ctypes.c_void_p(0x1000)
 

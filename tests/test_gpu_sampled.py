@@ -1,0 +1,129 @@
+"""spiffy_unmask_decide_sampled against the sampling oracle: drawn tokens bit
+for bit wherever the oracle's best and second best noisy scores are not within
+rounding of each other, confidences within tolerance, the rule's decision where
+its margin allows, and the losslessness invariant through the CUDA call."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import sampling as S
+from oracle import toy
+from paper_2509_18085_b200 import spiffy
+from paper_2509_18085_b200 import workloads as W
+import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+DRAW_GAP = 1e-4   # fp32 noise and scores against the oracle's float64
+
+
+def case(seed, B, N, L, V, dtype, p_unmasked=0.3):
+    r = np.random.default_rng(seed)
+    logits = W.round_to((r.standard_normal((B, N, L, V)) * 2).astype(np.float32), dtype)
+    mask = V - 1
+    logits[..., mask] = W.round_to(np.float32(-30.0), dtype)
+    tokens = np.where(r.random((B, N, L)) < p_unmasked, r.integers(0, V - 1, (B, N, L)), mask).astype(np.int32)
+    tokens[:, :, 0] = mask
+    return logits, tokens, mask
+
+
+def check(logits, tokens, mask, dtype, rule, top_s, tau, T, seed):
+    dec = spiffy.spiffy_unmask_decide_sampled(G.to_dev(logits, torch.bfloat16 if dtype == "bf16" else None),
+                                              G.to_dev(tokens), mask, rule, T, seed, top_s, tau)
+    torch.cuda.synchronize()
+    o = S.sampled_decide(logits, tokens, mask, rule, top_s, tau, T, seed)
+    sure = o.draw_gap > DRAW_GAP
+    got_tok = dec.top_tok.cpu().numpy()
+    assert np.array_equal(got_tok[sure], o.top_tok[sure])
+    assert sure.mean() > 0.99
+    masked = tokens == mask
+    ok = sure & masked
+    np.testing.assert_allclose(dec.conf.cpu().numpy()[ok], o.conf[ok], atol=G.TOL[dtype] if dtype == "bf16" else 1e-4)
+    assert np.all(np.isneginf(dec.conf.cpu().numpy()[~masked]))
+    assert np.array_equal(got_tok[~masked], tokens[~masked])
+    node_ok = sure.all(axis=2) & (o.margin > (1e-3 if dtype == "bf16" else 1e-4))
+    assert np.array_equal(G.bits_np(dec.unmask_bits)[node_ok], o.unmask_bits[node_ok])
+    assert np.array_equal(dec.n_unmask.cpu().numpy()[node_ok], o.n_unmask[node_ok])
+    if logits.shape[-1] <= 10000:  # with longer vocabularies the confidences are too close to compare the rule
+        assert node_ok.any()
+    assert int(dec.dev_status.sum()) == 0
+    return dec, o
+
+
+@pytest.mark.parametrize("dtype,V", [("bf16", 8192), ("bf16", 33000), ("f32", 4100), ("f32", 1001 * 4),
+                                     ("bf16", 126464), ("f32", 36), ("bf16", 8)])
+@pytest.mark.parametrize("T", [0.7, 1.0])
+def test_draws_match_the_oracle(dtype, V, T):
+    B, N, L = (1, 2, 5) if V > 100000 else (2, 3, 9)
+    logits, tokens, mask = case(V, B, N, L, V, dtype)
+    for rule, S_, tau in ((spiffy.RULE_TOPS, 2, 0.0), (spiffy.RULE_THRESHOLD, 1, 0.05)):
+        check(logits, tokens, mask, dtype, rule, S_, tau, T, seed=1234 + V)
+
+
+def test_noise_ignores_the_node_and_follows_the_seed_and_the_state():
+    logits, tokens, mask = case(3, 1, 1, 6, 5000, "f32", p_unmasked=0.0)
+    x = np.repeat(logits, 4, axis=1)
+    st = np.repeat(tokens, 4, axis=1)
+    st[0, 3, 2] = 17  # node 3 is one step further
+    run = lambda seed: spiffy.spiffy_unmask_decide_sampled(G.to_dev(x), G.to_dev(st), mask, spiffy.RULE_TOPS,
+                                                           1.0, seed).top_tok.cpu().numpy()
+    a, b, c = run(5), run(5), run(6)
+    assert np.array_equal(a, b)                       # deterministic
+    assert np.array_equal(a[0, 0], a[0, 1]) and np.array_equal(a[0, 0], a[0, 2])
+    assert not np.array_equal(a[0, 0], c[0, 0])       # another seed, other draws
+    keep = np.arange(6) != 2
+    assert not np.array_equal(a[0, 0][keep], a[0, 3][keep])  # another masked count, other noise
+
+
+def test_draw_frequencies_follow_the_tempered_softmax():
+    """One call with many sequences: each sequence index is part of the counter,
+    so the B draws of position 0 are independent samples of one distribution."""
+    B, V, T = 4000, 8, 1.3
+    x = np.array([1.0, 0.2, -0.5, 2.0, 0.0, 0.7, -1.0, -30.0], dtype=np.float32)
+    logits = np.broadcast_to(x, (B, 1, 1, V)).copy()
+    tokens = np.full((B, 1, 1), V - 1, dtype=np.int32)
+    dec = spiffy.spiffy_unmask_decide_sampled(G.to_dev(logits), G.to_dev(tokens), V - 1, spiffy.RULE_TOPS, T, 77)
+    tok = dec.top_tok.cpu().numpy().reshape(-1)
+    p = np.exp(x.astype(np.float64) / T)
+    p /= p.sum()
+    freq = np.bincount(tok, minlength=V) / B
+    assert np.all(np.abs(freq - p) < 4 * np.sqrt(p * (1 - p) / B) + 1e-9), (freq, p)
+    np.testing.assert_allclose(dec.conf.cpu().numpy().reshape(-1), p[tok], atol=1e-5)
+
+
+def test_argument_checks():
+    logits, tokens, mask = case(1, 1, 2, 4, 64, "f32")
+    lg, tk = G.to_dev(logits), G.to_dev(tokens)
+    for bad_t in (0.0, -1.0, float("nan"), float("inf")):
+        with pytest.raises(spiffy.SpiffyError):
+            spiffy.spiffy_unmask_decide_sampled(lg, tk, mask, spiffy.RULE_TOPS, bad_t, 1)
+    with pytest.raises(spiffy.SpiffyError):
+        spiffy.spiffy_unmask_decide_sampled(lg, tk, mask, spiffy.RULE_TOPS, 1.0, 1,
+                                            workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
+
+
+@pytest.mark.parametrize("seed", range(2))
+def test_sampled_decoding_through_the_cuda_call_is_lossless(seed):
+    """App. A at T = 1 with the CUDA sampled decision and the CUDA walk."""
+    def decide(logits, states, mask_id, rule, top_s, threshold):
+        d = spiffy.spiffy_unmask_decide_sampled(G.to_dev(logits), G.to_dev(states.astype(np.int32)), mask_id,
+                                                rule, 1.0, 900 + seed, top_s, threshold)
+        return d.top_tok.cpu().numpy(), G.bits_np(d.unmask_bits)
+
+    def walk(states, off, idx, top_tok, unmask_bits, mask_id):
+        g = spiffy.spiffy_accept_walk(G.to_dev(states.astype(np.int32)), G.to_dev(off), G.to_dev(idx),
+                                      G.to_dev(top_tok.astype(np.int32)), G.to_dev(unmask_bits.view(np.int64)))
+        return (g.accepted_node.cpu().numpy(), g.n_accepted.cpu().numpy(), g.path.cpu().numpy(),
+                g.next_block.cpu().numpy())
+
+    model = toy.ToyModel(seed=seed)
+    s0 = np.full(model.block_len, model.mask_id, dtype=np.int32)
+    s0[seed] = 2
+    vanilla = toy.vanilla_decode(model, s0, oracle.RULE_TOPS, decide=decide)
+    calls = model.calls
+    model.calls = 0
+    drafter = toy.peeking_drafter(vanilla, depth=3, wrong_prob=0.2, seed=seed, vocab=model.vocab)
+    traj, accepted = toy.speculative_decode(model, s0, drafter, oracle.RULE_TOPS, decide=decide, walk=walk)
+    assert len(traj) == len(vanilla) and all(np.array_equal(a, b) for a, b in zip(traj, vanilla))
+    assert model.calls == calls - sum(accepted) and sum(accepted) > 0
