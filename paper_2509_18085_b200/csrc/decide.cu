@@ -1,5 +1,5 @@
 // Decision kernels: steps 1-4 of Algorithm 1 (the function Next() of App. A)
-// evaluated for every node of the draft graph.
+// evaluated for every node of the draft graph, and their fusion with step 5.
 //
 //   decide_reduce_kernel    streams the logits rows of still-masked positions
 //                           once (the HBM-bound part): per (row, vocabulary
@@ -8,10 +8,12 @@
 //   decide_finalize_kernel  per node: merges the slices in a fixed order, turns
 //                           them into (confidence, top token) and applies the
 //                           unmasking rule of Sec. 3.1
+//   decide_tail_kernel      per sequence, for small graphs: the finalize step
+//                           of all its nodes and the acceptance walk (step 5)
+//                           in one CTA, resident before the reduce ends
 //
-// The argmax compares logit values exactly ((value desc, index asc) order);
-// probabilities only enter the confidence.  All merges run in a fixed order, so
-// repeated calls give identical bits.
+// The arithmetic shared with the other decision kernels is in decide_core.cuh,
+// the walk in walk_core.cuh.
 #include "common.cuh"
 #include "decide_core.cuh"
 #include "walk_core.cuh"
