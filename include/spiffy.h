@@ -405,7 +405,10 @@ size_t spiffy_draft_blocks_workspace(const spiffy_draft_desc* desc);
  *   state       [B][L] int32 current block
  *   formula_off [D+1], formula_i, formula_j: CSR of the (i, j) pairs, shared
  *               by all sequences; parents before children
- *   child_off   [D+1], child_idx: children of each formula in the draft graph
+ *   child_off   [D+1], child_idx: children of each formula in the draft graph.
+ *               These five arrays are constants of the model: they must be
+ *               complete in device memory before the call is made (the kernels
+ *               read them without waiting for earlier work on the stream)
  *   draft_tokens [B][D*+1][L]: node 0 = the current block, then the kept drafts
  *               in formula order; unused nodes repeat the current block
  *   kept        [B][D*] formula index of every kept draft, -1 for unused nodes

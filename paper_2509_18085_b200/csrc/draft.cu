@@ -82,6 +82,7 @@ draft_topk_kernel(const T* __restrict__ logits, int64_t row_stride, int V, int64
                   TopPartial* __restrict__ partials) {
 #if __CUDA_ARCH__ >= 900
   cudaGridDependencySynchronize();
+  pdl_launch_dependents();  // the build kernel (one CTA per sequence) may take its SM and stage the graph
 #endif
   const int row = blockIdx.y;
   if (state[row] != mask_id) return;
@@ -122,17 +123,31 @@ draft_topk_kernel(const T* __restrict__ logits, int64_t row_stride, int V, int64
   __shared__ float w_val[kThreads / 32];
   __shared__ int w_idx[kThreads / 32];
   __shared__ float w_sum[kThreads / 32];
+  // the thread's best remaining element; it is searched again only by the thread whose
+  // element has just been taken (every other thread's best is still its best)
+  float tv;
+  int ti;
+#define SPIFFY_DRAFT_RESCAN()                                                          \
+  do {                                                                                 \
+    tv = -INFINITY;                                                                    \
+    ti = 0x7fffffff;                                                                   \
+    _Pragma("unroll") for (int k = NE - 1; k >= 0; --k) /* descending: ties end on the lowest token */ \
+      if (x[k] >= tv && x[k] != -INFINITY) {                                           \
+        tv = x[k];                                                                     \
+        ti = index_of(k);                                                              \
+      }                                                                                \
+  } while (0)
+  SPIFFY_DRAFT_RESCAN();
   TopPartial out;
   out.s = 0.f;
-  float ml = 0.f;
+#pragma unroll
   for (int r = 0; r < kMaxK; ++r) {
     float bv = -INFINITY;
     int bi = 0x7fffffff;
     if (r < K) {
-      // the thread's best remaining element, then the CTA's
-#pragma unroll
-      for (int k = NE - 1; k >= 0; --k)
-        if (x[k] > bv || (x[k] == bv && x[k] != -INFINITY)) { bv = x[k]; bi = index_of(k); }
+      // the best remaining element of the CTA: the best over the threads
+      bv = tv;
+      bi = ti;
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) {
         const float v2 = __shfl_xor_sync(0xffffffffu, bv, off);
@@ -149,7 +164,7 @@ draft_topk_kernel(const T* __restrict__ logits, int64_t row_stride, int V, int64
         if (ahead(w_val[w], w_idx[w], bv, bi)) { bv = w_val[w]; bi = w_idx[w]; }
       if (r == 0) {
         // sum of exp(x - m) against the slice maximum, before anything is knocked out
-        ml = (bv == -INFINITY) ? 0.f : bv * kLog2e;
+        const float ml = (bv == -INFINITY) ? 0.f : bv * kLog2e;
         float s = 0.f;
 #pragma unroll
         for (int k = 0; k < NE; ++k) s += ex2(fmaf(x[k], kLog2e, -ml));
@@ -162,14 +177,17 @@ draft_topk_kernel(const T* __restrict__ logits, int64_t row_stride, int V, int64
         out.m = bv;
         out.s = s;
       }
-      // knock the winner out
+      if (bv != -INFINITY && ti == bi && r + 1 < K) {  // this thread's element was taken: knock it out, search again
 #pragma unroll
-      for (int k = 0; k < NE; ++k)
-        if (bv != -INFINITY && index_of(k) == bi) x[k] = -INFINITY;
+        for (int k = 0; k < NE; ++k)
+          if (index_of(k) == bi) x[k] = -INFINITY;
+        SPIFFY_DRAFT_RESCAN();
+      }
     }
     out.val[r] = bv;
     out.idx[r] = bv == -INFINITY ? 0x7fffffff : bi;
   }
+#undef SPIFFY_DRAFT_RESCAN
   out.pad[0] = out.pad[1] = 0;
   if (tid == 0) partials[(int64_t)row * splits + split] = out;
 }
@@ -210,9 +228,6 @@ __device__ bool strict_subset(const BuildArgs& g, int a, int c) {
 // grid = B sequences, 1024 threads; dynamic shared memory, see the carve-up below.
 __global__ void __launch_bounds__(kBuildThreads)
 draft_build_kernel(BuildArgs g) {
-#if __CUDA_ARCH__ >= 900
-  cudaGridDependencySynchronize();
-#endif
   const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int L = g.L, K = g.K, D = g.D;
   extern __shared__ __align__(8) unsigned char draft_smem[];
@@ -228,7 +243,9 @@ draft_build_kernel(BuildArgs g) {
   const int32_t* state = g.state + (int64_t)b * L;
   if (tid == 0) n_masked = 0;
   // The formulas are walked several times with dependent reads: when the graph
-  // fits, copy it to shared memory (the copy overlaps step 1) and walk it there.
+  // fits, copy it to shared memory and walk it there.  The draft graph is a
+  // constant of the model (calibrated offline), not the product of earlier work on
+  // the stream, so it is fetched before the wait on that work.
   __shared__ int32_t graph_smem[kGraphInts];
   {
     const int npairs = g.formula_off[D], nkids = g.child_off[D];
@@ -244,6 +261,9 @@ draft_build_kernel(BuildArgs g) {
       g.formula_off = f_off; g.child_off = c_off; g.formula_i = f_i; g.formula_j = f_j; g.child_idx = c_idx;
     }
   }
+#if __CUDA_ARCH__ >= 900
+  cudaGridDependencySynchronize();  // the top-k kernel's partial results, and the caller's logits and state, are visible
+#endif
   __syncthreads();
 
   // 1. candidates c_ij and their probabilities: one warp per position
