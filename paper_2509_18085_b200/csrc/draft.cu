@@ -274,12 +274,45 @@ draft_build_kernel(BuildArgs g) {
       continue;
     }
     const TopPartial* p = g.partials + ((int64_t)b * L + l) * g.splits;
-    // maximum and sum over the slices, fixed order
     float m = -INFINITY, s = 0.f;
-    for (int k = lane; k < g.splits; k += 32) {
-      const float m2 = p[k].m, s2 = p[k].s, M = fmaxf(m, m2);
-      s = s * ((m == M) ? 1.f : ex2((m - M) * kLog2e)) + s2 * ((m2 == M) ? 1.f : ex2((m2 - M) * kLog2e));
-      m = M;
+    float hv[kMaxK];
+    int hi[kMaxK];
+#pragma unroll
+    for (int t = 0; t < kMaxK; ++t) { hv[t] = -INFINITY; hi[t] = 0x7fffffff; }
+    if (g.splits <= 32) {
+      // one slice per lane, fetched whole in one trip: its maximum and sum, and its K
+      // candidates, which the top-k kernel left sorted
+      if (lane < g.splits) {
+        const uint4* q = reinterpret_cast<const uint4*>(p + lane);
+        const uint4 q0 = q[0], q1 = q[1], q2 = q[2];
+        m = __uint_as_float(q0.x);
+        s = __uint_as_float(q0.y);
+        hv[0] = __uint_as_float(q0.z); hv[1] = __uint_as_float(q0.w);
+        hv[2] = __uint_as_float(q1.x); hv[3] = __uint_as_float(q1.y);
+        hi[0] = (int)q1.z; hi[1] = (int)q1.w; hi[2] = (int)q2.x; hi[3] = (int)q2.y;
+#pragma unroll
+        for (int t = 0; t < kMaxK; ++t)
+          if (t >= K || hv[t] == -INFINITY) { hv[t] = -INFINITY; hi[t] = 0x7fffffff; }
+      }
+    } else {
+      // maximum and sum over the slices, fixed order
+      for (int k = lane; k < g.splits; k += 32) {
+        const float m2 = p[k].m, s2 = p[k].s, M = fmaxf(m, m2);
+        s = s * ((m == M) ? 1.f : ex2((m - M) * kLog2e)) + s2 * ((m2 == M) ? 1.f : ex2((m2 - M) * kLog2e));
+        m = M;
+      }
+      // every lane sorts the candidates it reads (each is read once)
+      for (int c = lane; c < g.splits * K; c += 32) {
+        float v = p[c / K].val[c % K];
+        int i = p[c / K].idx[c % K];
+        if (v == -INFINITY) continue;
+#pragma unroll
+        for (int t = 0; t < kMaxK; ++t)  // insertion into the sorted list
+          if (ahead(v, i, hv[t], hi[t])) {
+            const float tv = hv[t]; const int ti = hi[t];
+            hv[t] = v; hi[t] = i; v = tv; i = ti;
+          }
+      }
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
@@ -290,24 +323,8 @@ draft_build_kernel(BuildArgs g) {
     }
     if (lane == 0 && (!(fabsf(m) < INFINITY) || !(s > 0.f) || !(s < INFINITY)) && g.dev_status)
       atomicOr(g.dev_status + b, SPIFFY_DEV_NONFINITE);
-    // the K best of the splits * K slice candidates (value desc, id asc): every lane
-    // first sorts the candidates it reads (each is read once), then K rounds pick the
-    // best head over the lanes and pop it
-    float hv[kMaxK];
-    int hi[kMaxK];
-#pragma unroll
-    for (int t = 0; t < kMaxK; ++t) { hv[t] = -INFINITY; hi[t] = 0x7fffffff; }
-    for (int c = lane; c < g.splits * K; c += 32) {
-      float v = p[c / K].val[c % K];
-      int i = p[c / K].idx[c % K];
-      if (v == -INFINITY) continue;
-#pragma unroll
-      for (int t = 0; t < kMaxK; ++t)  // insertion into the sorted list
-        if (ahead(v, i, hv[t], hi[t])) {
-          const float tv = hv[t]; const int ti = hi[t];
-          hv[t] = v; hi[t] = i; v = tv; i = ti;
-        }
-    }
+    // the K best of the slices' candidates (value desc, id asc): K rounds pick the best
+    // head over the lanes and pop it
     for (int r = 0; r < K; ++r) {
       float bv = hv[0];
       int bi = hi[0];
@@ -412,31 +429,40 @@ draft_build_kernel(BuildArgs g) {
       tokens[n * L + l] = cand_tok[l * kMaxK + g.formula_j[e]];
     }
   }
-  // 7. parent lists: every earlier kept node whose candidate set is a strict subset
-  for (int c = tid; c <= g.budget; c += kBuildThreads) {
+  // 7. parent lists: every earlier kept node whose candidate set is a strict subset.
+  // One warp per child, its lanes over the candidate parents.
+  auto is_parent = [&](int a, int c) {
+    return a < c && (a == 0 || node_formula[a] >= 0) &&
+           strict_subset(g, a == 0 ? -1 : node_formula[a], node_formula[c]);
+  };
+  for (int c = warp; c <= g.budget; c += kBuildThreads / 32) {
     int n = 0;
     if (c > 0 && node_formula[c] >= 0)
-      for (int a = 0; a < c; ++a)
-        n += (a == 0 || node_formula[a] >= 0) && strict_subset(g, a == 0 ? -1 : node_formula[a], node_formula[c]);
-    n_parents[c] = n;
+      for (int a0 = 0; a0 < c; a0 += 32) n += __popc(__ballot_sync(0xffffffffu, is_parent(a0 + lane, c)));
+    if (lane == 0) n_parents[c] = n;
   }
   __syncthreads();
-  for (int c = tid; c <= g.budget; c += kBuildThreads) {
+  for (int c = warp; c <= g.budget; c += kBuildThreads / 32) {
     int start = 0;
-    for (int x = 0; x < c; ++x) start += n_parents[x];
+    for (int x = lane; x < c; x += 32) start += n_parents[x];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) start += __shfl_xor_sync(0xffffffffu, start, off);
     int32_t* off = g.parent_off + (int64_t)b * (g.budget + 2);
     int32_t* idx = g.parent_idx + (int64_t)b * g.parent_cap;
-    off[c] = min(start, g.parent_cap);
-    if (c == g.budget) off[c + 1] = min(start + n_parents[c], g.parent_cap);
-    if (start + n_parents[c] > g.parent_cap && g.dev_status) atomicOr(g.dev_status + b, SPIFFY_DEV_BADGRAPH);
+    if (lane == 0) {
+      off[c] = min(start, g.parent_cap);
+      if (c == g.budget) off[c + 1] = min(start + n_parents[c], g.parent_cap);
+      if (start + n_parents[c] > g.parent_cap && g.dev_status) atomicOr(g.dev_status + b, SPIFFY_DEV_BADGRAPH);
+    }
     if (c > 0 && node_formula[c] >= 0) {
       int w = start;
-      for (int a = 0; a < c; ++a)
-        if ((a == 0 || node_formula[a] >= 0) &&
-            strict_subset(g, a == 0 ? -1 : node_formula[a], node_formula[c])) {
-          if (w < g.parent_cap) idx[w] = a;
-          ++w;
-        }
+      for (int a0 = 0; a0 < c; a0 += 32) {
+        const bool par = is_parent(a0 + lane, c);
+        const unsigned mask = __ballot_sync(0xffffffffu, par);
+        const int at = w + __popc(mask & ((1u << lane) - 1u));
+        if (par && at < g.parent_cap) idx[at] = a0 + lane;
+        w += __popc(mask);
+      }
     }
   }
 }

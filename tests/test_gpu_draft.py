@@ -116,3 +116,17 @@ def test_nothing_left_to_draft_and_single_rank():
     assert_parity(got, want)
     assert got.kept[0].cpu().tolist() == [-1] * 5 and got.kept[1].cpu().tolist() == [0, 1, 2, 3, -1]
     assert torch.equal(got.tokens[0], torch.from_numpy(state[0]).cuda().expand(6, L))
+
+
+def test_more_than_32_vocabulary_slices():
+    """A vocabulary long enough (fp32, more than 32 slices of 4096) for the build
+    kernel's general slice merge, and all ten drafts kept (a parent list per node)."""
+    r = np.random.default_rng(3)
+    B, L, V = 2, 5, 140000
+    logits = (r.standard_normal((B, L, V)) * 3).astype(np.float32)
+    logits[..., V - 1] = -30.0
+    state = np.full((B, L), V - 1, dtype=np.int32)
+    state[1, 3] = 11
+    got, want = run_both(logits, state, V - 1, 10, 3, torch.float32)
+    assert assert_parity(got, want) == B
+    assert int(want.parent_off[0, -1]) > 10
