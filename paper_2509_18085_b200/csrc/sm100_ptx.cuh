@@ -61,7 +61,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
 }
-// 4-D tile load global -> shared (this CTA only, no multicast); completion is
+// 4-D tile load global -> shared, into this CTA alone; completion is
 // signalled on `bar` as transferred bytes.  c0 is the innermost coordinate and
 // must be a multiple of 8 for 16-bit elements.
 __device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* m, uint64_t* bar,
