@@ -22,6 +22,8 @@
  *                            nodes the walk reaches (fewer bytes read);
  *   spiffy_unmask_decide_sampled
  *                            steps 1-4 at sampling temperature T > 0;
+ *   spiffy_lmhead_decide     steps 1-4 fused into the output projection: the
+ *                            logits are reduced on the tensor cores, never stored;
  *   spiffy_draft_blocks      drafting and pruning (Sec. 4.4.2, Sec. 4.4.4): the
  *                            draft blocks and parent lists of the next step;
  *   spiffy_stage_masked_rows, spiffy_unmask_decide_static
@@ -259,6 +261,31 @@ spiffy_status spiffy_unmask_decide_sampled(const spiffy_decide_desc* desc,
                                            int32_t* n_unmask, int32_t* dev_status,
                                            void* workspace, size_t workspace_bytes,
                                            void* cuda_stream);
+
+/*
+ * Steps 1-4 of Algorithm 1 straight from the hidden states: the logits
+ *   x[r][v] = sum_k hidden_states[r][k] * weight[v][k]       (fp32 accumulation)
+ * are formed tile by tile on the tensor cores and reduced there, so that the
+ * [rows x V] logits are never written to memory; the result is what
+ * spiffy_unmask_decide gives on those (unrounded, fp32) logits.
+ *   hidden_states [B*N*L][hidden] bf16, row r = (b * N + n) * L + l; rows of
+ *                 unmasked positions are computed and ignored
+ *   weight        [V][hidden] bf16 (the output embedding, one row per token)
+ *   desc          batch, n_nodes, block_len, vocab, mask_token_id, rule, top_s,
+ *                 threshold are used; logits_dtype and row_stride are ignored
+ * Limits: B * N * L <= 256, hidden a multiple of 128; else SPIFFY_EUNSUPPORTED.
+ * Outputs, status bits and the finalize step are those of spiffy_unmask_decide.
+ * The paper evaluates the decision on materialised logits; fusing it into the
+ * output projection is this library's addition.
+ * Workspace: spiffy_lmhead_decide_workspace(desc, hidden) (depends on the
+ * device's SM count; 0 when the shape is not supported).
+ */
+size_t spiffy_lmhead_decide_workspace(const spiffy_decide_desc* desc, int32_t hidden);
+spiffy_status spiffy_lmhead_decide(const spiffy_decide_desc* desc, int32_t hidden,
+                                   const void* hidden_states, const void* weight,
+                                   const int32_t* block_tokens, float* conf, int32_t* top_tok,
+                                   uint64_t* unmask_bits, int32_t* n_unmask, int32_t* dev_status,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------- */
 /* Acceptance: step 5 of Algorithm 1 over the draft graph of Sec. 4.4.1      */

@@ -230,6 +230,49 @@ spiffy_status spiffy_unmask_decide_sampled(const spiffy_decide_desc* desc,
                                static_cast<cudaStream_t>(cuda_stream));
 }
 
+namespace {
+// The descriptor of the fused call names no logits: fill those fields in so that the
+// common checks apply.
+spiffy_status lmhead_desc(const spiffy_decide_desc* desc, int32_t hidden, spiffy_decide_desc* out) {
+  if (!desc) return SPIFFY_EINVAL;
+  *out = *desc;
+  out->logits_dtype = SPIFFY_BF16;
+  out->row_stride = ((int64_t)desc->vocab + 7) / 8 * 8;
+  const spiffy_status st = check_decide_desc(out, true);
+  if (st != SPIFFY_OK) return st;
+  if (hidden < 128 || hidden % 128 != 0) return SPIFFY_EUNSUPPORTED;
+  if ((int64_t)desc->batch * desc->n_nodes * desc->block_len > 256) return SPIFFY_EUNSUPPORTED;
+  return SPIFFY_OK;
+}
+}  // namespace
+
+size_t spiffy_lmhead_decide_workspace(const spiffy_decide_desc* desc, int32_t hidden) {
+  spiffy_decide_desc d;
+  if (lmhead_desc(desc, hidden, &d) != SPIFFY_OK) return 0;
+  const int grid = lmhead_grid(d);
+  return grid > 0 ? lmhead_workspace_bytes(d, grid) : 0;
+}
+
+spiffy_status spiffy_lmhead_decide(const spiffy_decide_desc* desc, int32_t hidden,
+                                   const void* hidden_states, const void* weight,
+                                   const int32_t* block_tokens, float* conf, int32_t* top_tok,
+                                   uint64_t* unmask_bits, int32_t* n_unmask, int32_t* dev_status,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  spiffy_decide_desc d;
+  const spiffy_status st = lmhead_desc(desc, hidden, &d);
+  if (st != SPIFFY_OK) return st;
+  if (!hidden_states || !weight || !block_tokens || !conf || !top_tok || !unmask_bits || !n_unmask)
+    return SPIFFY_EINVAL;
+  if (!aligned16(hidden_states) || !aligned16(weight)) return SPIFFY_EINVAL;
+  const int grid = lmhead_grid(d);
+  if (grid <= 0) return SPIFFY_ECUDA;
+  const size_t need = lmhead_workspace_bytes(d, grid);
+  if (!workspace || workspace_bytes < need || !aligned16(workspace)) return SPIFFY_EWORKSPACE;
+  return launch_lmhead_decide(d, hidden, hidden_states, weight, block_tokens, conf, top_tok,
+                              unmask_bits, n_unmask, dev_status, workspace,
+                              static_cast<cudaStream_t>(cuda_stream));
+}
+
 size_t spiffy_draft_blocks_workspace(const spiffy_draft_desc* desc) {
   if (check_draft_desc(desc) != SPIFFY_OK) return 0;
   return draft_workspace_bytes(*desc);

@@ -61,6 +61,17 @@ spiffy_status launch_decide_sampled(const spiffy_decide_desc& d, float temperatu
                                     int32_t* top_tok, uint64_t* unmask_bits, int32_t* n_unmask,
                                     int32_t* dev_status, void* ws, cudaStream_t stream);
 
+spiffy_status launch_decide_finalize(const spiffy_decide_desc& d, const void* partials, int splits,
+                                     const int32_t* block_tokens, float* conf, int32_t* top_tok,
+                                     uint64_t* unmask_bits, int32_t* n_unmask, int32_t* dev_status,
+                                     cudaStream_t stream);
+int lmhead_grid(const spiffy_decide_desc& d);
+size_t lmhead_workspace_bytes(const spiffy_decide_desc& d, int grid);
+spiffy_status launch_lmhead_decide(const spiffy_decide_desc& d, int hidden, const void* hstates,
+                                   const void* weight, const int32_t* block_tokens, float* conf,
+                                   int32_t* top_tok, uint64_t* unmask_bits, int32_t* n_unmask,
+                                   int32_t* dev_status, void* ws, cudaStream_t stream);
+
 spiffy_status launch_attention_simt(const spiffy_attn_desc& d, const void* q,
                                     const void* kp, const void* vp,
                                     const void* kb, const void* vb, void* out,

@@ -239,6 +239,22 @@ spiffy_status launch_decide(const spiffy_decide_desc& d, const void* logits,
   return e == cudaSuccess ? SPIFFY_OK : SPIFFY_ECUDA;
 }
 
+// The finalize kernel alone, on partial results another kernel produced
+// (`splits` per row, in the layout of this file's reduce kernel).
+spiffy_status launch_decide_finalize(const spiffy_decide_desc& d, const void* partials, int splits,
+                                     const int32_t* block_tokens, float* conf, int32_t* top_tok,
+                                     uint64_t* unmask_bits, int32_t* n_unmask, int32_t* dev_status,
+                                     cudaStream_t stream) {
+  const Partial* cpart = static_cast<const Partial*>(partials);
+  const cudaError_t e =
+      launch_pdl(decide_finalize_kernel, dim3(d.batch * d.n_nodes), dim3(kFinalizeThreads), (size_t)0,
+                 stream, cpart, splits, (int)d.n_nodes, (int)d.block_len, block_tokens,
+                 (int)d.mask_token_id, (int)d.rule, (int)d.top_s, d.threshold, conf, top_tok,
+                 unmask_bits, n_unmask, dev_status);
+  count_launch();
+  return e == cudaSuccess ? SPIFFY_OK : SPIFFY_ECUDA;
+}
+
 // Decision and walk in one call.  Small graphs (at most kTailRows rows per
 // sequence, arrays within the default shared-memory limit) take the fused tail:
 // two launches instead of three.  Larger ones keep one finalize CTA per node,

@@ -108,6 +108,10 @@ def lib() -> ctypes.CDLL:
         L.spiffy_unmask_decide_sampled.restype = ctypes.c_int
         L.spiffy_unmask_decide_sampled.argtypes = [ctypes.POINTER(DecideDesc), ctypes.POINTER(SampleDesc)] + \
             [vp] * 8 + [sz, vp]
+        L.spiffy_lmhead_decide_workspace.restype = sz
+        L.spiffy_lmhead_decide_workspace.argtypes = [ctypes.POINTER(DecideDesc), i32]
+        L.spiffy_lmhead_decide.restype = ctypes.c_int
+        L.spiffy_lmhead_decide.argtypes = [ctypes.POINTER(DecideDesc), i32] + [vp] * 9 + [sz, vp]
         L.spiffy_status_string.restype = ctypes.c_char_p
         L.spiffy_status_string.argtypes = [ctypes.c_int]
         L.spiffy_launch_count.restype = ctypes.c_uint64
@@ -274,6 +278,45 @@ def spiffy_unmask_decide_sampled(logits, block_tokens, mask_token_id: int, rule:
         _dev(out.dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
         workspace.numel() * workspace.element_size(), _stream(stream))
     _check(st, "spiffy_unmask_decide_sampled")
+    return out
+
+
+def spiffy_lmhead_decide(hidden_states, weight, block_tokens, mask_token_id: int, rule: int,
+                         top_s: int = 1, threshold: float = 0.9, out: Optional[Decision] = None,
+                         workspace=None, stream=None) -> Decision:
+    """Steps 1-4 of Algorithm 1 straight from the hidden states: logits =
+    hidden_states @ weight.T are formed and reduced on the tensor cores without
+    ever being written.  hidden_states [B,N,L,H] bf16 (B*N*L <= 256, H a multiple
+    of 128), weight [V,H] bf16, block_tokens [B,N,L] int32."""
+    B, N, L = block_tokens.shape
+    H = hidden_states.shape[-1]
+    V = weight.shape[0]
+    if hidden_states.dtype != torch.bfloat16 or weight.dtype != torch.bfloat16:
+        raise ValueError("hidden_states and weight must be bf16")
+    if tuple(hidden_states.shape) != (B, N, L, H) or weight.shape[1] != H:
+        raise ValueError("hidden_states must be [B,N,L,H] and weight [V,H]")
+    if not hidden_states.is_contiguous() or not weight.is_contiguous():
+        raise ValueError("hidden_states and weight must be contiguous")
+    desc = DecideDesc(B, N, L, V, BF16, V, int(mask_token_id), int(rule), int(top_s), float(threshold))
+    dev = hidden_states.device
+    if out is None:
+        out = Decision(torch.empty((B, N, L), dtype=torch.float32, device=dev),
+                       torch.empty((B, N, L), dtype=torch.int32, device=dev),
+                       torch.empty((B, N), dtype=torch.int64, device=dev),
+                       torch.empty((B, N), dtype=torch.int32, device=dev),
+                       torch.zeros((B,), dtype=torch.int32, device=dev))
+    if workspace is None:
+        need = int(lib().spiffy_lmhead_decide_workspace(ctypes.byref(desc), int(H)))
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    st = lib().spiffy_lmhead_decide(
+        ctypes.byref(desc), int(H), _dev(hidden_states, "hidden_states"), _dev(weight, "weight"),
+        _dev(block_tokens, "block_tokens", torch.int32),
+        _dev(out.conf, "conf", torch.float32), _dev(out.top_tok, "top_tok", torch.int32),
+        _dev(out.unmask_bits, "unmask_bits", torch.int64),
+        _dev(out.n_unmask, "n_unmask", torch.int32),
+        _dev(out.dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
+        workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(st, "spiffy_lmhead_decide")
     return out
 
 

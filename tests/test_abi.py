@@ -177,6 +177,24 @@ def test_sampled_decide_rejects_bad_arguments(lib):
         spiffy.EUNSUPPORTED
 
 
+def test_lmhead_decide_rejects_bad_arguments(lib):
+    fake = ctypes.c_void_p(0x1000)
+    good = spiffy.DecideDesc(1, 8, 32, 126464, 0, 0, 126463, spiffy.RULE_THRESHOLD, 1, 0.9)
+
+    def call(d=good, hidden=4096, hs=fake, w=fake):
+        return lib.spiffy_lmhead_decide(ctypes.byref(d), hidden, hs, w, fake, fake, fake, fake, fake, None,
+                                        fake, 1 << 30, None)
+
+    assert call(hidden=100) == spiffy.EUNSUPPORTED          # not a multiple of 128
+    assert call(hidden=0) == spiffy.EUNSUPPORTED
+    assert call(d=spiffy.DecideDesc(1, 9, 32, 1000, 0, 0, 999, spiffy.RULE_TOPS, 1, 0.0)) == spiffy.EUNSUPPORTED
+    assert call(d=spiffy.DecideDesc(1, 8, 32, 0, 0, 0, 0, spiffy.RULE_TOPS, 1, 0.0)) == spiffy.EINVAL
+    assert call(d=spiffy.DecideDesc(1, 8, 32, 1000, 0, 0, 999, 9, 1, 0.0)) == spiffy.EINVAL
+    assert call(hs=None) == spiffy.EINVAL
+    assert call(w=ctypes.c_void_p(0x1008)) == spiffy.EINVAL
+    assert lib.spiffy_lmhead_decide_workspace(ctypes.byref(good), 100) == 0
+
+
 def test_draft_rejects_bad_arguments(lib):
     fake = ctypes.c_void_p(0x1000)
 
