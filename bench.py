@@ -56,7 +56,7 @@ def parse():
     ap.add_argument("--nodes", type=int, default=None, help="node count for configuration 5")
     ap.add_argument("--attn-kernel", default="auto", choices=["auto", "simt", "tcgen05"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--part", default="step", choices=["step", "attention", "decide", "decide_walk", "decide_walk_lazy", "decide_sampled", "draft"],
+    ap.add_argument("--part", default="step", choices=["step", "attention", "decide", "decide_walk", "decide_walk_lazy", "decide_sampled", "lmhead", "draft"],
                     help="time one library call alone on any configuration (for profiling); "
                          "the benchmark line itself is --part step")
     ap.add_argument("--sets", type=int, default=0, help="rotating input sets for --part (0 = enough to exceed L2)")
@@ -233,6 +233,8 @@ def run_part(args):
     cfg = W.config(args.config, args.nodes)
     if args.part == "draft":
         return run_draft_part(args, cfg)
+    if args.part == "lmhead":
+        return run_lmhead_part(args, cfg)
     attn = args.part == "attention"
     probe = W.make(cfg, W.seed_for(args.config, 100), attention=attn, decision=not attn)
     masked = int((probe.block_tokens == cfg.mask_id).sum())
@@ -294,6 +296,49 @@ def run_part(args):
                        note="gbs counts the eager call's bytes (every node); lazy_gbs the bytes this call reads")
     out["peaks"] = peaks["source"]
     print(json.dumps(out))
+
+
+def run_lmhead_part(args, cfg):
+    """spiffy_lmhead_decide alone: the decision fused into the output projection
+    at the configuration's rows and vocabulary, hidden size 4096 (LLaDA-8B),
+    random bf16 operands.  The 1 GB weight matrix is larger than L2 by itself."""
+    import ctypes
+    import torch
+    from paper_2509_18085_b200 import spiffy
+    hidden = 4096
+    B, N, L, V = cfg.batch, cfg.n_nodes, cfg.block_len, cfg.vocab
+    g = torch.Generator().manual_seed(11)
+    hs = torch.randn((B, N, L, hidden), generator=g).to(torch.bfloat16).cuda()
+    w = (torch.randn((V, hidden), generator=g) * (2.0 / hidden ** 0.5)).to(torch.bfloat16).cuda()
+    tokens = torch.where(torch.rand((B, N, L), generator=g) < 0.36, 3, cfg.mask_id).to(torch.int32).cuda()
+    desc = spiffy.DecideDesc(B, N, L, V, spiffy.BF16, V, cfg.mask_id, cfg.rule, cfg.top_s, cfg.threshold)
+    ws = torch.empty(int(spiffy.lib().spiffy_lmhead_decide_workspace(ctypes.byref(desc), hidden)),
+                     dtype=torch.uint8, device="cuda")
+    call = lambda out=None: spiffy.spiffy_lmhead_decide(hs, w, tokens, cfg.mask_id, cfg.rule, cfg.top_s,
+                                                        cfg.threshold, out=out, workspace=ws)
+    out = call()
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for _ in range(max(3, args.warmup // 10)):
+            call(out)
+        stream.synchronize()
+        reps = max(5, args.steps // 100)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            call(out)
+        e1.record(stream)
+        stream.synchronize()
+        sec = e0.elapsed_time(e1) * 1e-3 / reps
+    peaks = measured_peaks()
+    flops = 2.0 * B * N * L * V * hidden
+    by = (V + B * N * L) * hidden * 2.0
+    print(json.dumps({"part": "lmhead", "config": f"config{args.config}-{cfg.name}", "us_per_call": sec * 1e6,
+                      "rows": B * N * L, "hidden": hidden, "vocab": V, "calls_timed": reps,
+                      "tflops": flops / sec / 1e12, "frac_of_bf16_peak": flops / sec / 1e12 / peaks["bf16_tflops"],
+                      "gbs": by / sec / 1e9, "frac_of_hbm": by / sec / 1e9 / peaks["hbm_gbs"],
+                      "algorithmic_flops": flops, "algorithmic_bytes": by, "peaks": peaks["source"],
+                      "dev_status": int(out.dev_status.max().item())}))
 
 
 def run_draft_part(args, cfg):
