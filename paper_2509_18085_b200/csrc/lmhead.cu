@@ -37,7 +37,7 @@ using namespace sm100;
 constexpr int kLmThreads = 320;
 constexpr int kLmStages = 3;
 constexpr int kTile = 128 * 128;        // one operand tile of a stage: 128 rows x 64 bf16 = 16 KB
-constexpr int kLmN = 256;               // vocabulary entries per tile
+constexpr int kLmN = 256;               // most vocabulary entries per tile
 constexpr int kStageBytes = 4 * kTile;  // H tile 0 | H tile 1 | W tile (256 rows)
 constexpr int kLmBars = 2 * kLmStages + 4;
 constexpr int kLmSmem = kLmStages * kStageBytes + 8 * kLmBars + 16 + 1024;
@@ -45,6 +45,7 @@ constexpr uint32_t kLmTmemCols = 512;   // M-tile t -> columns 256 t .. 256 t + 
 
 struct LmParams {
   int rows, hidden, vocab, mt;  // mt = M-tiles (1 or 2)
+  int n_tile;                   // vocabulary entries per tile: a multiple of 32, at most kLmN
   Partial* partials;            // [rows][gridDim.x]
   int32_t* status;              // [B], may be null
   int n_status;
@@ -65,7 +66,7 @@ lmhead_reduce_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_cons
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_tiles = (p.vocab + kLmN - 1) / kLmN;
+  const int n_tiles = (p.vocab + p.n_tile - 1) / p.n_tile;
   const int my_tiles = (int)blockIdx.x < n_tiles ? (n_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
   const int kc_count = p.hidden / 64;
 
@@ -98,11 +99,11 @@ lmhead_reduce_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_cons
           const int stage = it % kLmStages;
           if (!mbar_wait(empty + stage, (((uint32_t)(it / kLmStages)) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t* dst = smem + stage * kStageBytes;
-          mbar_arrive_expect_tx(full + stage, (uint32_t)(p.mt + 2) * kTile);
+          mbar_arrive_expect_tx(full + stage, (uint32_t)p.mt * kTile + (uint32_t)p.n_tile * 128u);
           const int c0 = (kc & 1) * 64, head = kc >> 1;
           tma_load_4d(dst, &tm_h, full + stage, c0, head, 0, 0);
           if (p.mt > 1) tma_load_4d(dst + kTile, &tm_h, full + stage, c0, head, 128, 0);
-          tma_load_4d(dst + 2 * kTile, &tm_w, full + stage, c0, head, n * kLmN, 0);
+          tma_load_4d(dst + 2 * kTile, &tm_w, full + stage, c0, head, n * p.n_tile, 0);
           issued = it + 1;
         }
       }
@@ -115,7 +116,7 @@ lmhead_reduce_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_cons
   } else if (warp == 1) {
     // ---------------------------------------------------------- MMA issuer --
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16_f32(128, kLmN, false, false);
+      const uint32_t idesc = idesc_bf16_f32(128, p.n_tile, false, false);
       bool ok = true;
       int it = 0;
       for (int i = 0; i < my_tiles && ok; ++i) {
@@ -160,10 +161,10 @@ lmhead_reduce_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_cons
         tc_fence_after_sync();
         const uint32_t col0 = (uint32_t)t * (uint32_t)kLmN;
 #pragma unroll 1
-        for (int c0 = 0; c0 < kLmN; c0 += 32) {
+        for (int c0 = 0; c0 < p.n_tile; c0 += 32) {
           uint32_t v[32];
           tmem_ld_x32(tmem_addr(tmem, lane_base, col0 + (uint32_t)c0), v);
-          const int v0 = n * kLmN + c0;
+          const int v0 = n * p.n_tile + c0;
           float cm = -INFINITY;
 #pragma unroll
           for (int c = 0; c < 32; ++c) {
@@ -210,6 +211,23 @@ lmhead_reduce_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_cons
 
 }  // namespace
 
+// Vocabulary entries per tile: the multiple of 32 (at most 256, at least 128) for which
+// rounds of tiles x tile width is smallest -- a narrower tile can fill the last round.
+int lmhead_tile(int vocab, int sms) {
+  int best = kLmN;
+  int64_t best_cost = -1;
+  for (int n = kLmN; n >= 128; n -= 32) {
+    const int64_t tiles = (vocab + n - 1) / n;
+    const int64_t rounds = (tiles + sms - 1) / sms;
+    const int64_t cost = rounds * (n + 64);  // a tile costs about its width plus a fixed part
+    if (best_cost < 0 || cost < best_cost) {
+      best = n;
+      best_cost = cost;
+    }
+  }
+  return best;
+}
+
 int lmhead_grid(const spiffy_decide_desc& d) {
   static int sms[64];
   int device = 0;
@@ -217,7 +235,8 @@ int lmhead_grid(const spiffy_decide_desc& d) {
   if (sms[device] == 0 &&
       cudaDeviceGetAttribute(&sms[device], cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
     return 0;
-  const int n_tiles = (d.vocab + kLmN - 1) / kLmN;
+  const int n = lmhead_tile(d.vocab, sms[device]);
+  const int n_tiles = (d.vocab + n - 1) / n;
   return n_tiles < sms[device] ? n_tiles : sms[device];
 }
 
@@ -232,9 +251,14 @@ spiffy_status launch_lmhead_decide(const spiffy_decide_desc& d, int hidden, cons
   const int rows = d.batch * d.n_nodes * d.block_len;
   const int grid = lmhead_grid(d);
   if (grid <= 0) return SPIFFY_ECUDA;
+  int sm_count = 0, dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return SPIFFY_ECUDA;
+  const int n_tile = lmhead_tile(d.vocab, sm_count);
   CUtensorMap tm_h, tm_w;
   if (!make_map(&tm_h, hstates, hidden / 128, rows, 1, 1, 128) ||
-      !make_map(&tm_w, weight, hidden / 128, d.vocab, 1, 1, kLmN))
+      !make_map(&tm_w, weight, hidden / 128, d.vocab, 1, 1, n_tile))
     return SPIFFY_ECUDA;
   static bool attr_set[64];
   int device = 0;
@@ -250,6 +274,7 @@ spiffy_status launch_lmhead_decide(const spiffy_decide_desc& d, int hidden, cons
   p.hidden = hidden;
   p.vocab = d.vocab;
   p.mt = (rows + 127) / 128;
+  p.n_tile = n_tile;
   p.partials = static_cast<Partial*>(ws);
   p.status = dev_status;
   p.n_status = d.batch;
