@@ -273,7 +273,9 @@ spiffy_status spiffy_unmask_decide_sampled(const spiffy_decide_desc* desc,
  *   weight        [V][hidden] bf16 (the output embedding, one row per token)
  *   desc          batch, n_nodes, block_len, vocab, mask_token_id, rule, top_s,
  *                 threshold are used; logits_dtype and row_stride are ignored
- * Limits: B * N * L <= 256, hidden a multiple of 128; else SPIFFY_EUNSUPPORTED.
+ * Limit: hidden a multiple of 128, else SPIFFY_EUNSUPPORTED.  Rows are taken 256 at a
+ * time and every such pass reads the weight matrix again: the call is made for
+ * the few hundred rows of one verification step.
  * Outputs, status bits and the finalize step are those of spiffy_unmask_decide.
  * The paper evaluates the decision on materialised logits; fusing it into the
  * output projection is this library's addition.

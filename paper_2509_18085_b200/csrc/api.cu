@@ -241,7 +241,6 @@ spiffy_status lmhead_desc(const spiffy_decide_desc* desc, int32_t hidden, spiffy
   const spiffy_status st = check_decide_desc(out, true);
   if (st != SPIFFY_OK) return st;
   if (hidden < 128 || hidden % 128 != 0) return SPIFFY_EUNSUPPORTED;
-  if ((int64_t)desc->batch * desc->n_nodes * desc->block_len > 256) return SPIFFY_EUNSUPPORTED;
   return SPIFFY_OK;
 }
 }  // namespace

@@ -4,10 +4,11 @@
 // never written to memory (Algorithm 1, steps 1-2, on the distribution of
 // Sec. 3.1 before it is materialised).
 //
-// H: [rows][hidden] bf16 hidden states of the B*N*L positions (rows <= 256),
+// H: [rows][hidden] bf16 hidden states of the B*N*L positions,
 // W: [vocabulary][hidden] bf16 output embedding.  A CTA owns vocabulary tiles of
-// 256 entries (tile n, n + grid, ...), both M-tiles of 128 rows at once, and
-// runs the K loop over `hidden` in chunks of 64:
+// up to 256 entries (tile n, n + grid, ...), two M-tiles of 128 rows at once, and
+// runs the K loop over `hidden` in chunks of 64 (more than 256 rows are taken 256
+// at a time, each pass reading the weight matrix again):
 //   warp 0      TMA producer: per chunk the two H tiles and the W tile (64 KB)
 //               into a three-stage ring
 //   warp 1      allocates tensor memory; one lane issues tcgen05.mma, M = 128,
@@ -44,7 +45,7 @@ constexpr int kLmSmem = kLmStages * kStageBytes + 8 * kLmBars + 16 + 1024;
 constexpr uint32_t kLmTmemCols = 512;   // M-tile t -> columns 256 t .. 256 t + 255
 
 struct LmParams {
-  int rows, hidden, vocab, mt;  // mt = M-tiles (1 or 2)
+  int rows, hidden, vocab;
   int n_tile;                   // vocabulary entries per tile: a multiple of 32, at most kLmN
   Partial* partials;            // [rows][gridDim.x]
   int32_t* status;              // [B], may be null
@@ -69,11 +70,12 @@ lmhead_reduce_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_cons
   const int n_tiles = (p.vocab + p.n_tile - 1) / p.n_tile;
   const int my_tiles = (int)blockIdx.x < n_tiles ? (n_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
   const int kc_count = p.hidden / 64;
+  const int passes = (p.rows + 255) / 256;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kLmStages; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, 1); }
     mbar_init(acc_full, 1);
-    mbar_init(acc_empty, 128u * (uint32_t)p.mt);
+    mbar_init(acc_empty, 256u);  // every epilogue thread, also those of an M-tile beyond the rows
     *abort_flag = 0;
     mbar_fence_init();
   }
@@ -93,16 +95,18 @@ lmhead_reduce_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_cons
     if (lane == 0) {
       bool ok = true;
       int it = 0, issued = 0;
-      for (int i = 0; i < my_tiles && ok; ++i) {
+      for (int g = 0; g < passes * my_tiles && ok; ++g) {
+        const int pass = g / my_tiles, i = g - pass * my_tiles;
         const int n = (int)blockIdx.x + i * (int)gridDim.x;
+        const int row0 = pass * 256, mt = p.rows - row0 > 128 ? 2 : 1;
         for (int kc = 0; kc < kc_count; ++kc, ++it) {
           const int stage = it % kLmStages;
           if (!mbar_wait(empty + stage, (((uint32_t)(it / kLmStages)) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t* dst = smem + stage * kStageBytes;
-          mbar_arrive_expect_tx(full + stage, (uint32_t)p.mt * kTile + (uint32_t)p.n_tile * 128u);
+          mbar_arrive_expect_tx(full + stage, (uint32_t)mt * kTile + (uint32_t)p.n_tile * 128u);
           const int c0 = (kc & 1) * 64, head = kc >> 1;
-          tma_load_4d(dst, &tm_h, full + stage, c0, head, 0, 0);
-          if (p.mt > 1) tma_load_4d(dst + kTile, &tm_h, full + stage, c0, head, 128, 0);
+          tma_load_4d(dst, &tm_h, full + stage, c0, head, row0, 0);
+          if (mt > 1) tma_load_4d(dst + kTile, &tm_h, full + stage, c0, head, row0 + 128, 0);
           tma_load_4d(dst + 2 * kTile, &tm_w, full + stage, c0, head, n * p.n_tile, 0);
           issued = it + 1;
         }
@@ -119,8 +123,9 @@ lmhead_reduce_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_cons
       const uint32_t idesc = idesc_bf16_f32(128, p.n_tile, false, false);
       bool ok = true;
       int it = 0;
-      for (int i = 0; i < my_tiles && ok; ++i) {
-        if (!mbar_wait(acc_empty, ((uint32_t)i & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+      for (int g = 0; g < passes * my_tiles && ok; ++g) {
+        const int mt = p.rows - (g / my_tiles) * 256 > 128 ? 2 : 1;
+        if (!mbar_wait(acc_empty, ((uint32_t)g & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after_sync();
         for (int kc = 0; kc < kc_count; ++kc, ++it) {
           const int stage = it % kLmStages;
@@ -130,7 +135,7 @@ lmhead_reduce_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_cons
           const uint32_t w0 = h0 + 2 * kTile;
 #pragma unroll
           for (int t = 0; t < 2; ++t) {
-            if (t < p.mt) {
+            if (t < mt) {
               const uint32_t d = tmem + (uint32_t)t * (uint32_t)kLmN;
 #pragma unroll
               for (int kk = 0; kk < 4; ++kk)
@@ -147,21 +152,23 @@ lmhead_reduce_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_cons
     // ------------------------------------------------------------ epilogue --
     const int quad = warp & 3;
     const int t = (warp - 2) >> 2;  // M-tile of this warpgroup
-    if (t < p.mt) {
-      const int r = quad * 32 + lane;
-      const int row = t * 128 + r;
-      const uint32_t lane_base = (uint32_t)(quad * 32);
+    const int r = quad * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(quad * 32);
+    bool ok = true;
+    for (int pass = 0; pass < passes && ok; ++pass) {
+      const int row = pass * 256 + t * 128 + r;
+      const bool live = pass * 256 + t * 128 < p.rows;  // this warpgroup's M-tile holds rows in this pass
       float m_run = -INFINITY, s_run = 0.f, best = -INFINITY;
       int best_idx = 0x7fffffff;
-      bool ok = true;
       for (int i = 0; i < my_tiles && ok; ++i) {
         const int n = (int)blockIdx.x + i * (int)gridDim.x;
-        ok = __all_sync(0xffffffffu, mbar_wait(acc_full, (uint32_t)i & 1u, abort_flag));
+        const int g = pass * my_tiles + i;
+        ok = __all_sync(0xffffffffu, mbar_wait(acc_full, (uint32_t)g & 1u, abort_flag));
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t col0 = (uint32_t)t * (uint32_t)kLmN;
 #pragma unroll 1
-        for (int c0 = 0; c0 < p.n_tile; c0 += 32) {
+        for (int c0 = 0; live && c0 < p.n_tile; c0 += 32) {
           uint32_t v[32];
           tmem_ld_x32(tmem_addr(tmem, lane_base, col0 + (uint32_t)c0), v);
           const int v0 = n * p.n_tile + c0;
@@ -190,7 +197,7 @@ lmhead_reduce_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_cons
         tc_fence_before_sync();
         mbar_arrive(acc_empty);
       }
-      if (row < p.rows) {
+      if (ok && row < p.rows) {
         // NaN logits never win a comparison: report them through the maximum
         if (!(s_run == s_run)) m_run = s_run;
         p.partials[(int64_t)row * gridDim.x + blockIdx.x] =
@@ -273,7 +280,6 @@ spiffy_status launch_lmhead_decide(const spiffy_decide_desc& d, int hidden, cons
   p.rows = rows;
   p.hidden = hidden;
   p.vocab = d.vocab;
-  p.mt = (rows + 127) / 128;
   p.n_tile = n_tile;
   p.partials = static_cast<Partial*>(ws);
   p.status = dev_status;

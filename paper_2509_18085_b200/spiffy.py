@@ -286,8 +286,8 @@ def spiffy_lmhead_decide(hidden_states, weight, block_tokens, mask_token_id: int
                          workspace=None, stream=None) -> Decision:
     """Steps 1-4 of Algorithm 1 straight from the hidden states: logits =
     hidden_states @ weight.T are formed and reduced on the tensor cores without
-    ever being written.  hidden_states [B,N,L,H] bf16 (B*N*L <= 256, H a multiple
-    of 128), weight [V,H] bf16, block_tokens [B,N,L] int32."""
+    ever being written.  hidden_states [B,N,L,H] bf16 (H a multiple of 128),
+    weight [V,H] bf16, block_tokens [B,N,L] int32."""
     B, N, L = block_tokens.shape
     H = hidden_states.shape[-1]
     V = weight.shape[0]

@@ -187,7 +187,7 @@ def test_lmhead_decide_rejects_bad_arguments(lib):
 
     assert call(hidden=100) == spiffy.EUNSUPPORTED          # not a multiple of 128
     assert call(hidden=0) == spiffy.EUNSUPPORTED
-    assert call(d=spiffy.DecideDesc(1, 9, 32, 1000, 0, 0, 999, spiffy.RULE_TOPS, 1, 0.0)) == spiffy.EUNSUPPORTED
+    assert call(d=spiffy.DecideDesc(1, 9, 65, 1000, 0, 0, 999, spiffy.RULE_TOPS, 1, 0.0)) == spiffy.EUNSUPPORTED
     assert call(d=spiffy.DecideDesc(1, 8, 32, 0, 0, 0, 0, spiffy.RULE_TOPS, 1, 0.0)) == spiffy.EINVAL
     assert call(d=spiffy.DecideDesc(1, 8, 32, 1000, 0, 0, 999, 9, 1, 0.0)) == spiffy.EINVAL
     assert call(hs=None) == spiffy.EINVAL
