@@ -100,7 +100,7 @@ typedef enum { SPIFFY_RULE_TOPS = 0, SPIFFY_RULE_THRESHOLD = 1 } spiffy_rule;
 typedef struct {
   int32_t batch;      /* B >= 1                                              */
   int32_t n_nodes;    /* N >= 1                                              */
-  int32_t block_len;  /* L in [1, 64]                                        */
+  int32_t block_len;  /* L in [1, 1024]; [1, 64] on the CUDA-core kernel        */
   int32_t prefix_len; /* P >= 0 context keys shared by all nodes             */
   int32_t n_q_heads;  /* Hq                                                  */
   int32_t n_kv_heads; /* Hkv, divides Hq; query head h reads kv head

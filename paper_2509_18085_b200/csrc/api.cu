@@ -22,7 +22,7 @@ spiffy_status check_attn_desc(const spiffy_attn_desc* d) {
   if (d->dtype != SPIFFY_F32 && d->dtype != SPIFFY_BF16) return SPIFFY_EINVAL;
   if (!(d->scale >= 0.f) || !(d->scale < INFINITY)) return SPIFFY_EINVAL;
   if (d->kernel < SPIFFY_ATTN_AUTO || d->kernel > SPIFFY_ATTN_TCGEN05) return SPIFFY_EINVAL;
-  if (d->block_len > 64) return SPIFFY_EUNSUPPORTED;
+  if (d->block_len > 1024) return SPIFFY_EUNSUPPORTED;
   if (d->head_dim != 64 && d->head_dim != 128) return SPIFFY_EUNSUPPORTED;
   if (d->n_nodes > 65535 || d->batch > 65535) return SPIFFY_EUNSUPPORTED;
   return SPIFFY_OK;
@@ -98,6 +98,7 @@ spiffy_status spiffy_graph_attention(const spiffy_attn_desc* desc, const void* q
                                dev_status, workspace, stream);
   }
   if (d.kernel == SPIFFY_ATTN_TCGEN05) return SPIFFY_EUNSUPPORTED;
+  if (d.block_len > 64) return SPIFFY_EUNSUPPORTED;  // the CUDA-core kernel keeps a block's rows in registers
   return launch_attention_simt(d, q, k_prefix, v_prefix, k_block, v_block, out, stream);
 }
 
