@@ -199,6 +199,34 @@ def spiffy_unmask_decide_workspace(desc: DecideDesc) -> int:
     return int(lib().spiffy_unmask_decide_workspace(ctypes.byref(desc)))
 
 
+def spiffy_full_sequence_attention(q_nodes, q_suffix, k_prefix, v_prefix, k_suffix, v_suffix, k_block,
+                                   v_block, scale: float = 0.0, stream=None):
+    """The verification attention of a full-sequence bidirectional model that
+    caches only its prefix (Fig. 3 caption, App. A.2): the block being decoded
+    (node 0) and the trailing masked blocks attend to the whole true sequence,
+    every draft block to the prefix, the trailing blocks and itself.  Two calls
+    of spiffy_graph_attention on the tensor-core kernel:
+      nodes   context = [prefix ; suffix], blocks = the N node blocks;
+      suffix  one node whose block is the suffix, context = [prefix ; true block].
+    q_nodes [B,N,L,Hq,d], q_suffix [B,S,Hq,d], k/v_prefix [B,P,Hkv,d], k/v_suffix
+    [B,S,Hkv,d], k/v_block [B,N,L,Hkv,d], all bf16, d = 128, S <= 1024.  The two
+    contexts are assembled with torch.cat here; a caller that keeps its cache as
+    [suffix | prefix | true block] can pass views to the two calls instead.
+    Returns (out_nodes [B,N,L,Hq,d], out_suffix [B,S,Hq,d])."""
+    B, S = q_suffix.shape[0], q_suffix.shape[1]
+    ctx_nodes_k = torch.cat([k_prefix, k_suffix], 1) if k_prefix is not None else k_suffix.contiguous()
+    ctx_nodes_v = torch.cat([v_prefix, v_suffix], 1) if v_prefix is not None else v_suffix.contiguous()
+    out_nodes = spiffy_graph_attention(q_nodes, ctx_nodes_k, ctx_nodes_v, k_block, v_block, scale=scale,
+                                       kernel=ATTN_TCGEN05, stream=stream)
+    true_k, true_v = k_block[:, 0], v_block[:, 0]
+    ctx_suffix_k = torch.cat([k_prefix, true_k], 1) if k_prefix is not None else true_k.contiguous()
+    ctx_suffix_v = torch.cat([v_prefix, true_v], 1) if v_prefix is not None else true_v.contiguous()
+    out_suffix = spiffy_graph_attention(q_suffix.unsqueeze(1).contiguous(), ctx_suffix_k, ctx_suffix_v,
+                                        k_suffix.unsqueeze(1).contiguous(), v_suffix.unsqueeze(1).contiguous(),
+                                        scale=scale, kernel=ATTN_TCGEN05, stream=stream)
+    return out_nodes, out_suffix.squeeze(1)
+
+
 @dataclass
 class Decision:
     conf: torch.Tensor         # [B,N,L] float32
