@@ -229,7 +229,7 @@ spiffy_status spiffy_unmask_decide_static(const spiffy_decide_desc* desc,
                                           void* cuda_stream);
 
 /*
- * The decision step at sampling temperature T > 0 (Sec. 5.4 runs Spiffy at
+ * The decision step at sampling temperature T > 0 (Sec. 5.3, "Effect of Temperature", runs Spiffy at
  * T > 0; the sampler itself is not given in the paper and is fixed here).
  * Per still-masked position the token is drawn from softmax(x / T) as
  *   top_tok = argmax_v (x_v / T + g_v),  g_v = -ln(-ln u_v)      (Gumbel-max)
@@ -314,6 +314,13 @@ spiffy_status spiffy_lmhead_decide(const spiffy_decide_desc* desc, int32_t hidde
  *   dev_status    [B] OR-ed with SPIFFY_DEV_BADGRAPH when an offset or index is
  *                 out of range (such entries are ignored); may be NULL
  * Uses desc->batch, n_nodes, block_len only.
+ * Ordering: block_tokens and the parent lists (here, in spiffy_decide_walk and in
+ * the lazy call) are fetched while earlier work of the stream may still be
+ * draining.  They must be complete in memory before the kernel that precedes
+ * this call in the stream can let its dependents start, which holds for every
+ * kernel of this library and for any kernel that does not use programmatic
+ * dependent launch; do not produce them with an early-triggering kernel of your
+ * own placed directly before the call.
  */
 spiffy_status spiffy_accept_walk(const spiffy_decide_desc* desc,
                                  const int32_t* block_tokens,
@@ -361,10 +368,15 @@ spiffy_status spiffy_decide_walk(const spiffy_decide_desc* desc, const void* log
  *   - walk_status reports a malformed parent list only if the walk scanned it;
  *     SPIFFY_DEV_TIMEOUT in both status words when a bounded wait between the
  *     levels ran out (results are then unspecified).
- * Each level costs two grid-wide barriers, so the call pays off when one
- * node's share of the logits is large (long vocabularies, batches) and loses
- * to spiffy_decide_walk on a single short graph.  SPIFFY_EUNSUPPORTED when
- * the batch exceeds the number of thread blocks the device holds at once.
+ * There is no grid-wide barrier: per sequence, the thread blocks that reduce
+ * the current node's rows count themselves in on an arrival counter, the block
+ * that owns the sequence waits for that count, decides, and publishes the next
+ * node under an epoch number the reducers wait for; sequences never wait for one
+ * another.  A level still costs two such round trips through memory, so the
+ * call pays off when one node's share of the logits is large (long
+ * vocabularies, batches) and loses to spiffy_decide_walk on a single short
+ * graph.  SPIFFY_EUNSUPPORTED when the batch exceeds the number of thread blocks
+ * the device holds at once.
  * Workspace: spiffy_decide_walk_lazy_workspace(desc); contents on entry
  * arbitrary (the call zeroes the few bytes it needs with a memset on the
  * stream).
@@ -457,6 +469,27 @@ spiffy_status spiffy_draft_blocks(const spiffy_draft_desc* desc, const void* log
                                   int32_t* parent_off, int32_t* parent_idx,
                                   int32_t* dev_status, void* workspace,
                                   size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Failure-detection hook (the paper has no counterpart).  Every device-side wait
+ * of this library is bounded: an mbarrier wait of the tensor-core kernels gives
+ * up after a number of polls, a wait on a global-memory word of
+ * spiffy_decide_walk_lazy likewise; the kernel then sets SPIFFY_DEV_TIMEOUT in
+ * the caller's status word(s), lets copies in flight land, frees its tensor
+ * memory and returns, so the context stays usable.  This call changes those
+ * limits for all later launches of the process, so that a test can make a wait
+ * run out without hanging or faulting anything:
+ *   mbarrier_polls       polls per mbarrier wait; 0 = give up without waiting
+ *                        (the kernel then issues no copy it does not wait for
+ *                        and no tensor-core product); < 0 restores the default
+ *   flag_polls           polls (about 100 ns apart) per wait of the lazy call;
+ *                        < 0 restores the default
+ *   lazy_extra_arrivals  sequence 0 of the lazy call waits for this many
+ *                        arrivals more than can come (0 = normal operation)
+ * Values above the defaults are clamped to them.  Not for production use.
+ */
+void spiffy_set_wait_limits(int64_t mbarrier_polls, int64_t flag_polls,
+                            int32_t lazy_extra_arrivals);
 
 /* Static description of a status code; never NULL. */
 const char* spiffy_status_string(spiffy_status status);

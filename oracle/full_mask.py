@@ -17,11 +17,19 @@ and the mask, written out here as a boolean matrix:
 Plain numpy in float64 with the mask materialised; nothing in the product
 package imports this module and it imports nothing from it.
 
+blockwise_causal_attention is the same packed call for block-causal models
+(last sentence of the caption of Fig. 3, App. A.2): a block attends to the
+blocks before it and to itself, never forward, so for the block being decoded
+the mask keeps the earlier blocks and the node's own block and hides every later
+block of the sequence.
+
 Pins (tests/test_oracle_full_mask.py): the node rows equal the packed-attention
 oracle with the suffix appended to the context; the suffix rows equal a library
 scaled-dot-product attention over the true sequence; without a suffix the result
 is the packed-attention oracle's; a draft's output does not change when the true
-block's keys do.
+block's keys do.  Block-causal variant: each node's rows equal a library
+scaled-dot-product attention with a block-causal mask over the sequence in
+which that node stands in place of the block being decoded.
 """
 from __future__ import annotations
 
@@ -68,3 +76,37 @@ def full_sequence_attention(q_nodes, q_suffix, k_prefix, v_prefix, k_suffix, v_s
     out_nodes[:, 0] = out[:, :L]
     out_nodes[:, 1:] = out[:, L + S:].reshape(B, N - 1, L, Hq, d)
     return out_nodes, out[:, L:L + S]
+
+
+def blockwise_causal_attention(q_nodes, k_seq, v_seq, k_block, v_block, block_index, scale=None):
+    """Verification attention of a block-causal model for block ``block_index``.
+    q_nodes [B,N,L,Hq,d]; k_seq, v_seq [B,n_blocks*L,Hkv,d]: keys and values of
+    the whole sequence (what is stored for blocks >= block_index is never
+    visible); k/v_block [B,N,L,Hkv,d]: the nodes' own blocks.  Returns
+    [B,N,L,Hq,d]."""
+    f = lambda a: np.asarray(a, dtype=np.float64)
+    q_nodes, k_seq, v_seq, k_block, v_block = f(q_nodes), f(k_seq), f(v_seq), f(k_block), f(v_block)
+    B, N, L, Hq, d = q_nodes.shape
+    T, Hkv = k_seq.shape[1], k_seq.shape[2]
+    rep = Hq // Hkv
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    # key axis: the sequence | block of node 0 | block of node 1 | ...
+    keys = np.concatenate([k_seq, k_block.reshape(B, N * L, Hkv, d)], 1)
+    vals = np.concatenate([v_seq, v_block.reshape(B, N * L, Hkv, d)], 1)
+    mask = np.zeros((N * L, T + N * L), dtype=bool)
+    for n in range(N):
+        rows = slice(n * L, (n + 1) * L)
+        for j in range(T):
+            mask[rows, j] = (j // L) < block_index            # earlier blocks only: never forward
+        mask[rows, T + n * L:T + (n + 1) * L] = True            # the node's own block, both directions
+    qs = q_nodes.reshape(B, N * L, Hq, d)
+    out = np.empty((B, N * L, Hq, d))
+    for b in range(B):
+        for h in range(Hq):
+            g = h // rep
+            s = (qs[b, :, h] @ keys[b, :, g].T) * scale
+            s = np.where(mask, s, -np.inf)
+            p = np.exp(s - s.max(axis=1, keepdims=True))
+            p /= p.sum(axis=1, keepdims=True)
+            out[b, :, h] = p @ vals[b, :, g]
+    return out.reshape(B, N, L, Hq, d)

@@ -1,7 +1,7 @@
 """CPU oracle of the decision step at sampling temperature T > 0 -- TEST
 INFRASTRUCTURE ONLY.
 
-The paper evaluates Spiffy at temperatures above zero (Sec. 5.4, SDAR at T = 1)
+The paper evaluates Spiffy at temperatures above zero (Sec. 5.3, SDAR at T = 1)
 without spelling the sampler out; the reading taken here (listed with the
 others in the design notes):
 

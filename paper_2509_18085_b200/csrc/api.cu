@@ -9,6 +9,14 @@ namespace spiffy {
 static std::atomic<uint64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
+// defaults: 2^20 mbarrier polls; 2^21 polls of about 100 ns each on a global word
+static std::atomic<uint32_t> g_mbar_polls{1u << 20};
+static std::atomic<uint32_t> g_flag_polls{1u << 21};
+static std::atomic<int32_t> g_lazy_extra{0};
+uint32_t mbar_poll_limit() { return g_mbar_polls.load(std::memory_order_relaxed); }
+uint32_t flag_poll_limit() { return g_flag_polls.load(std::memory_order_relaxed); }
+int32_t lazy_extra_arrivals() { return g_lazy_extra.load(std::memory_order_relaxed); }
+
 namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -309,6 +317,14 @@ const char* spiffy_status_string(spiffy_status status) {
     case SPIFFY_ECUDA: return "CUDA runtime error at launch";
   }
   return "unknown status";
+}
+
+void spiffy_set_wait_limits(int64_t mbarrier_polls, int64_t flag_polls, int32_t lazy_extra_arrivals) {
+  g_mbar_polls.store(mbarrier_polls < 0 ? (1u << 20) : (uint32_t)(mbarrier_polls > (1 << 20) ? (1 << 20) : mbarrier_polls),
+                     std::memory_order_relaxed);
+  g_flag_polls.store(flag_polls < 0 ? (1u << 21) : (uint32_t)(flag_polls > (1 << 21) ? (1 << 21) : flag_polls),
+                     std::memory_order_relaxed);
+  g_lazy_extra.store(lazy_extra_arrivals < 0 ? 0 : lazy_extra_arrivals, std::memory_order_relaxed);
 }
 
 uint64_t spiffy_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

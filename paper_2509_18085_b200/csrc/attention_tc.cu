@@ -91,13 +91,8 @@ struct Params {
   float* part_o;   // [splits][B*Hkv][MT][128][128]
   float* part_ml;  // [splits][B*Hkv][MT][128][2]
   int32_t* status;
+  uint32_t spin_limit;  // polls of one mbarrier wait
 };
-
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
@@ -207,7 +202,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         const uint32_t round = (uint32_t)(j / (is_k ? KS : VS));
         uint64_t* empty = (is_k ? k_empty : v_empty) + stage;
         uint64_t* full = (is_k ? k_full : v_full) + stage;
-        if (!mbar_wait(empty, (round & 1u) ^ 1u, abort_flag)) { ok = false; return; }
+        if (!mbar_wait(empty, (round & 1u) ^ 1u, abort_flag, p.spin_limit)) { ok = false; return; }
         const int t = t_begin + j;
         const bool ctx = t < p.TP;
         const CUtensorMap* m = is_k ? (ctx ? &tm_kp : &tm_kb) : (ctx ? &tm_vp : &tm_vb);
@@ -237,7 +232,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     if (lane == 0 && T > 0) {
       constexpr uint32_t idesc_s = idesc_bf16_f32(BM, BN, false, false);
       constexpr uint32_t idesc_o = idesc_bf16_f32(BM, HD, false, true);
-      bool ok = mbar_wait(q_full, 0, abort_flag);
+      bool ok = mbar_wait(q_full, 0, abort_flag, p.spin_limit);
       // S = Q K^T of key tile j into S buffer `buf`, from Q tile `qt`
       auto issue_s = [&](int j, int buf, int qt) {
         const uint32_t q_addr = smem_u32(sq + qt * kTileBytes);
@@ -264,7 +259,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         umma_commit(pv_done + buf);
       };
       auto wait_k = [&](int j) {
-        if (ok && !mbar_wait(k_full + j % KS, (uint32_t)(j / KS) & 1u, abort_flag)) ok = false;
+        if (ok && !mbar_wait(k_full + j % KS, (uint32_t)(j / KS) & 1u, abort_flag, p.spin_limit)) ok = false;
         tc_fence_after_sync();
       };
       if constexpr (NQ == 1) {
@@ -278,8 +273,8 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         s_tile(0);
         if (T > 1) s_tile(1);
         for (int j = 0; j < T && ok; ++j) {
-          if (!mbar_wait(p_ready + (j & 1), (uint32_t)(j >> 1) & 1u, abort_flag)) { ok = false; break; }
-          if (!mbar_wait(v_full + j % VS, (uint32_t)(j / VS) & 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(p_ready + (j & 1), (uint32_t)(j >> 1) & 1u, abort_flag, p.spin_limit)) { ok = false; break; }
+          if (!mbar_wait(v_full + j % VS, (uint32_t)(j / VS) & 1u, abort_flag, p.spin_limit)) { ok = false; break; }
           tc_fence_after_sync();
           issue_pv(j, j & 1, j < 2);
           umma_commit(v_empty + j % VS);
@@ -294,10 +289,10 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
           umma_commit(k_empty + 0);
         }
         for (int j = 0; j < T && ok; ++j) {
-          if (!mbar_wait(v_full + j % VS, (uint32_t)(j / VS) & 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(v_full + j % VS, (uint32_t)(j / VS) & 1u, abort_flag, p.spin_limit)) { ok = false; break; }
           if (j + 1 < T) wait_k(j + 1);
           for (int q = 0; q < 2 && ok; ++q) {
-            if (!mbar_wait(p_ready + q, (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(p_ready + q, (uint32_t)j & 1u, abort_flag, p.spin_limit)) { ok = false; break; }
             tc_fence_after_sync();
             issue_pv(j, q, j == 0);
             if (j + 1 < T) issue_s(j + 1, q, q);  // after PV: P of this tile has been consumed
@@ -337,7 +332,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
       const uint32_t col_s = kColS + (uint32_t)bi * BN;
       const uint32_t col_o = kColO + (uint32_t)bi * HD;
       // wait outcomes are made warp-uniform: the TMEM accesses below are warp-collective
-      if (!__all_sync(0xffffffffu, mbar_wait(s_full + bi, (uint32_t)mine & 1u, abort_flag))) {
+      if (!__all_sync(0xffffffffu, mbar_wait(s_full + bi, (uint32_t)mine & 1u, abort_flag, p.spin_limit))) {
         ok = false;
         break;
       }
@@ -379,7 +374,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         }
         if (mine > 0) {  // the accumulator holds this warpgroup's earlier tiles: wait, then rescale
           if (!__all_sync(0xffffffffu,
-                          mbar_wait(pv_done + bi, (uint32_t)(mine - 1) & 1u, abort_flag))) {
+                          mbar_wait(pv_done + bi, (uint32_t)(mine - 1) & 1u, abort_flag, p.spin_limit))) {
             ok = false;
             break;
           }
@@ -432,10 +427,10 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     // columns of every row.
     if (ok && mine > 0)
       ok = __all_sync(0xffffffffu,
-                      mbar_wait(pv_done + buf_hand, (uint32_t)(mine - 1) & 1u, abort_flag));
+                      mbar_wait(pv_done + buf_hand, (uint32_t)(mine - 1) & 1u, abort_flag, p.spin_limit));
     if (ok && solo && mine_alt > 0)
       ok = __all_sync(0xffffffffu, mbar_wait(pv_done + (buf_hand ^ 1), (uint32_t)(mine_alt - 1) & 1u,
-                                             abort_flag));
+                                             abort_flag, p.spin_limit));
     if constexpr (NQ == 2) {
       // each warpgroup owns its rows outright: normalise (or hand on the partial) and store
       if (ok) {
@@ -724,6 +719,7 @@ spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q, cons
   p.part_o = static_cast<float*>(ws);
   p.part_ml = p.part_o ? p.part_o + (size_t)pl.splits * pl.tiles * BM * HD : nullptr;
   p.status = dev_status;
+  p.spin_limit = mbar_poll_limit();
 
   if (cudaFuncSetAttribute(graph_attention_tc_kernel<1>,
                            cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||

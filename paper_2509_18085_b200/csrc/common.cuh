@@ -11,8 +11,31 @@ namespace spiffy {
 
 constexpr float kLog2e = 1.4426950408889634f;
 
+// 2^x on the special-function unit (approximate, denormals flushed).
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// 128-bit streaming load: read-only path, no L1 allocation (data used once).
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
 // Every launch of the library goes through this counter (spiffy_launch_count).
 void count_launch(int n = 1);
+
+// Poll limits of the bounded device-side waits, read at launch.  The defaults
+// (about a fraction of a second) change only through spiffy_set_wait_limits,
+// which exists so that the give-up paths can be exercised.
+uint32_t mbar_poll_limit();   // polls of one mbarrier wait (tensor-core kernels)
+uint32_t flag_poll_limit();   // polls of one wait on a global-memory word (lazy call)
+int32_t lazy_extra_arrivals();  // arrivals sequence 0's tail expects beyond those that can come
 
 // Entry points implemented in the kernel files; all validated by the caller.
 spiffy_status launch_decide(const spiffy_decide_desc& d, const void* logits,
@@ -96,8 +119,13 @@ spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q,
 
 // Launch with programmatic stream serialisation: the kernel may be scheduled
 // while its predecessor in the stream is still draining.  Every kernel launched
-// this way calls cudaGridDependencySynchronize() before it touches global
-// memory, so its reads and writes are ordered after the predecessor.
+// this way calls cudaGridDependencySynchronize() before it writes global memory
+// or reads what the calls of one step hand to each other (logits, partial
+// results, top tokens, unmask sets).  The walk, tail and draft-build kernels
+// fetch the graph arrays (block states, parent lists, draft formulas) ahead of
+// that wait: those must be complete before the predecessor can trigger its
+// dependents, which the library's own kernels guarantee (each waits for its
+// predecessor before it triggers) and the header states for callers.
 template <typename... Args>
 cudaError_t launch_pdl(void (*kern)(Args...), dim3 grid, dim3 block, size_t smem,
                        cudaStream_t stream, Args... args) {

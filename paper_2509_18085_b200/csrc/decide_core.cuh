@@ -29,12 +29,6 @@ struct __align__(16) Partial {
   int pad;
 };
 
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
 // Two fp32 lanes in one 64-bit register: Blackwell issues their multiply-add and
 // their add as one instruction each (the kernel is bound by instruction issue).
 __device__ __forceinline__ uint64_t pack2(float lo, float hi) {
@@ -61,14 +55,6 @@ __device__ __forceinline__ uint64_t add_exp2(uint64_t acc, float x0, float x1, u
   float a0, a1;
   unpack2(fma2(pack2(x0, x1), k2, nml2), a0, a1);
   return add2(acc, pack2(ex2(a0), ex2(a1)));
-}
-
-__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
-  return v;
 }
 
 // (value desc, index asc) merge of two partial results.

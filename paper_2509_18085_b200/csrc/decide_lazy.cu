@@ -57,9 +57,10 @@ struct LazyParams {
   int32_t* epoch;      // [B] levels of b whose tail has finished
   int32_t* cur;        // [B] node b stands on at level epoch[b], -1 once its walk has ended
   int stage_graph;     // the sequence's states and parent lists fit shared memory
+  unsigned wait_spins;   // polls of one wait before it gives up
+  unsigned extra_arrivals;  // test hook: sequence 0 expects this many arrivals that never come
 };
 
-constexpr unsigned kWaitSpins = 1u << 21;  // x ~100 ns: gives up after a fraction of a second
 
 __device__ __forceinline__ unsigned ld_acquire_u32(const void* p) {
   unsigned v;
@@ -69,13 +70,14 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const void* p) {
 
 // Thread 0 waits until the word at `p` has reached `target`; every thread of
 // the CTA gets the verdict (false: the wait ran out, here or elsewhere).
-__device__ __forceinline__ bool wait_reached(const void* p, unsigned target, LazyHeader* h) {
+__device__ __forceinline__ bool wait_reached(const void* p, unsigned target, LazyHeader* h,
+                                             unsigned limit) {
   __shared__ int ok_flag;
   if (threadIdx.x == 0) {
     unsigned spins = 0;
     bool ok = true;
     while (ld_acquire_u32(p) < target) {
-      if (++spins > kWaitSpins || *reinterpret_cast<volatile int*>(&h->timeout)) {
+      if (++spins > limit || *reinterpret_cast<volatile int*>(&h->timeout)) {
         ok = false;
         h->timeout = 1;
         break;
@@ -134,7 +136,8 @@ decide_walk_lazy_kernel(const LazyParams p) {
   if (tid == 0) s_bad = 0;
   int own_node = b_own >= 0 ? 0 : -1;  // uniform over the CTA
   int own_hops = 0;
-  unsigned own_expected = 0;           // arrivals[b_own] once the current level is reduced
+  // arrivals[b_own] once the current level is reduced
+  unsigned own_expected = b_own == 0 ? p.extra_arrivals : 0u;
   bool failed = false;
   const int items = p.B * L * p.splits;
   for (int level = 0; level < N && !failed; ++level) {
@@ -149,7 +152,7 @@ decide_walk_lazy_kernel(const LazyParams p) {
         if (b == b_own) {
           node = own_node;
         } else {
-          if (!wait_reached(p.epoch + b, (unsigned)level, p.header)) {
+          if (!wait_reached(p.epoch + b, (unsigned)level, p.header, p.wait_spins)) {
             failed = true;
             break;
           }
@@ -188,7 +191,7 @@ decide_walk_lazy_kernel(const LazyParams p) {
         for (int off = 16; off > 0; off >>= 1) masked += __shfl_xor_sync(0xffffffffu, masked, off);
         own_expected += (unsigned)masked * (unsigned)p.splits;
       }
-      if (!wait_reached(p.arrivals + b, own_expected, p.header)) {
+      if (!wait_reached(p.arrivals + b, own_expected, p.header, p.wait_spins)) {
         failed = true;
         break;
       }
@@ -355,6 +358,8 @@ spiffy_status launch_decide_walk_lazy(const spiffy_decide_desc& d, const void* l
   p.epoch = reinterpret_cast<int32_t*>(p.arrivals + d.batch);
   p.cur = p.epoch + d.batch;
   p.stage_graph = stage_graph;
+  p.wait_spins = flag_poll_limit();
+  p.extra_arrivals = (unsigned)lazy_extra_arrivals();
   const int64_t items = (int64_t)d.batch * d.block_len * p.splits;
   int grid = (int)(items < resident ? items : resident);
   if (grid < d.batch) grid = d.batch;

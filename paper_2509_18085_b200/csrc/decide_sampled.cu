@@ -1,4 +1,4 @@
-// Decision step at sampling temperature T > 0 (Sec. 5.4 evaluates Spiffy at
+// Decision step at sampling temperature T > 0 (Sec. 5.3 evaluates Spiffy at
 // T > 0; the paper does not spell the sampler out).
 //
 // Per still-masked position the token is drawn from softmax(x / T) by the

@@ -50,6 +50,7 @@ struct LmParams {
   Partial* partials;            // [rows][gridDim.x]
   int32_t* status;              // [B], may be null
   int n_status;
+  uint32_t spin_limit;          // polls of one mbarrier wait
 };
 
 __global__ void __launch_bounds__(kLmThreads, 1)
@@ -101,7 +102,7 @@ lmhead_reduce_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_cons
         const int row0 = pass * 256, mt = p.rows - row0 > 128 ? 2 : 1;
         for (int kc = 0; kc < kc_count; ++kc, ++it) {
           const int stage = it % kLmStages;
-          if (!mbar_wait(empty + stage, (((uint32_t)(it / kLmStages)) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(empty + stage, (((uint32_t)(it / kLmStages)) & 1u) ^ 1u, abort_flag, p.spin_limit)) { ok = false; break; }
           uint8_t* dst = smem + stage * kStageBytes;
           mbar_arrive_expect_tx(full + stage, (uint32_t)mt * kTile + (uint32_t)p.n_tile * 128u);
           const int c0 = (kc & 1) * 64, head = kc >> 1;
@@ -125,11 +126,11 @@ lmhead_reduce_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_cons
       int it = 0;
       for (int g = 0; g < passes * my_tiles && ok; ++g) {
         const int mt = p.rows - (g / my_tiles) * 256 > 128 ? 2 : 1;
-        if (!mbar_wait(acc_empty, ((uint32_t)g & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(acc_empty, ((uint32_t)g & 1u) ^ 1u, abort_flag, p.spin_limit)) { ok = false; break; }
         tc_fence_after_sync();
         for (int kc = 0; kc < kc_count; ++kc, ++it) {
           const int stage = it % kLmStages;
-          if (!mbar_wait(full + stage, (uint32_t)(it / kLmStages) & 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(full + stage, (uint32_t)(it / kLmStages) & 1u, abort_flag, p.spin_limit)) { ok = false; break; }
           tc_fence_after_sync();
           const uint32_t h0 = smem_u32(smem + stage * kStageBytes);
           const uint32_t w0 = h0 + 2 * kTile;
@@ -163,7 +164,7 @@ lmhead_reduce_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_cons
       for (int i = 0; i < my_tiles && ok; ++i) {
         const int n = (int)blockIdx.x + i * (int)gridDim.x;
         const int g = pass * my_tiles + i;
-        ok = __all_sync(0xffffffffu, mbar_wait(acc_full, (uint32_t)g & 1u, abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(acc_full, (uint32_t)g & 1u, abort_flag, p.spin_limit));
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t col0 = (uint32_t)t * (uint32_t)kLmN;
@@ -284,6 +285,7 @@ spiffy_status launch_lmhead_decide(const spiffy_decide_desc& d, int hidden, cons
   p.partials = static_cast<Partial*>(ws);
   p.status = dev_status;
   p.n_status = d.batch;
+  p.spin_limit = mbar_poll_limit();
   cudaError_t e = launch_pdl(lmhead_reduce_kernel, dim3(grid), dim3(kLmThreads), (size_t)kLmSmem, stream,
                              tm_h, tm_w, p);
   count_launch();

@@ -23,12 +23,6 @@ RULE_TOPS, RULE_THRESHOLD = 0, 1
 DEV_NONFINITE, DEV_BADGRAPH, DEV_TIMEOUT = 1, 2, 4
 ATTN_AUTO, ATTN_SIMT, ATTN_TCGEN05 = 0, 1, 2
 
-EXPORTS = (
-    "spiffy_graph_attention_workspace", "spiffy_graph_attention",
-    "spiffy_unmask_decide_workspace", "spiffy_unmask_decide",
-    "spiffy_accept_walk", "spiffy_status_string", "spiffy_launch_count",
-    "spiffy_unmask_decide_static", "spiffy_draft_blocks_workspace", "spiffy_draft_blocks",
-)
 DECIDE_STATIC_BYTES = 2 << 20
 
 
@@ -116,12 +110,21 @@ def lib() -> ctypes.CDLL:
         L.spiffy_status_string.argtypes = [ctypes.c_int]
         L.spiffy_launch_count.restype = ctypes.c_uint64
         L.spiffy_launch_count.argtypes = []
+        L.spiffy_set_wait_limits.restype = None
+        L.spiffy_set_wait_limits.argtypes = [ctypes.c_int64, ctypes.c_int64, i32]
         _lib = L
     return _lib
 
 
 def launch_count() -> int:
     return int(lib().spiffy_launch_count())
+
+
+def set_wait_limits(mbarrier_polls: int = -1, flag_polls: int = -1, lazy_extra_arrivals: int = 0):
+    """Failure-detection hook (spiffy_set_wait_limits): lowers the poll limits of
+    the library's bounded device-side waits so that a test can see one run out;
+    called without arguments it restores the defaults."""
+    lib().spiffy_set_wait_limits(int(mbarrier_polls), int(flag_polls), int(lazy_extra_arrivals))
 
 
 def _dtype_code(t: torch.Tensor) -> int:
@@ -258,11 +261,7 @@ def spiffy_unmask_decide(logits, block_tokens, mask_token_id: int, rule: int,
     B, N, L = block_tokens.shape
     dev = logits.device
     if out is None:
-        out = Decision(torch.empty((B, N, L), dtype=torch.float32, device=dev),
-                       torch.empty((B, N, L), dtype=torch.int32, device=dev),
-                       torch.empty((B, N), dtype=torch.int64, device=dev),
-                       torch.empty((B, N), dtype=torch.int32, device=dev),
-                       torch.zeros((B,), dtype=torch.int32, device=dev))
+        out = _new_decision(B, N, L, dev)
     need = spiffy_unmask_decide_workspace(desc)
     if workspace is None:
         workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
@@ -289,11 +288,7 @@ def spiffy_unmask_decide_sampled(logits, block_tokens, mask_token_id: int, rule:
     B, N, L = block_tokens.shape
     dev = logits.device
     if out is None:
-        out = Decision(torch.empty((B, N, L), dtype=torch.float32, device=dev),
-                       torch.empty((B, N, L), dtype=torch.int32, device=dev),
-                       torch.empty((B, N), dtype=torch.int64, device=dev),
-                       torch.empty((B, N), dtype=torch.int32, device=dev),
-                       torch.zeros((B,), dtype=torch.int32, device=dev))
+        out = _new_decision(B, N, L, dev)
     if workspace is None:
         need = int(lib().spiffy_unmask_decide_sampled_workspace(ctypes.byref(desc)))
         workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
@@ -328,11 +323,7 @@ def spiffy_lmhead_decide(hidden_states, weight, block_tokens, mask_token_id: int
     desc = DecideDesc(B, N, L, V, BF16, V, int(mask_token_id), int(rule), int(top_s), float(threshold))
     dev = hidden_states.device
     if out is None:
-        out = Decision(torch.empty((B, N, L), dtype=torch.float32, device=dev),
-                       torch.empty((B, N, L), dtype=torch.int32, device=dev),
-                       torch.empty((B, N), dtype=torch.int64, device=dev),
-                       torch.empty((B, N), dtype=torch.int32, device=dev),
-                       torch.zeros((B,), dtype=torch.int32, device=dev))
+        out = _new_decision(B, N, L, dev)
     if workspace is None:
         need = int(lib().spiffy_lmhead_decide_workspace(ctypes.byref(desc), int(H)))
         workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
@@ -383,11 +374,7 @@ def spiffy_accept_walk(block_tokens, parent_off, parent_idx, top_tok, unmask_bit
     dev = block_tokens.device
     desc = DecideDesc(B, N, L, 0, F32, 0, 0, 0, 1, 0.0)
     if out is None:
-        out = Walk(torch.empty((B,), dtype=torch.int32, device=dev),
-                   torch.empty((B,), dtype=torch.int32, device=dev),
-                   torch.empty((B, N), dtype=torch.int32, device=dev),
-                   torch.empty((B, L), dtype=torch.int32, device=dev),
-                   torch.zeros((B,), dtype=torch.int32, device=dev))
+        out = _new_walk(B, N, L, dev)
     if tuple(parent_off.shape) != (B, N + 1) or parent_idx.dim() != 2 or parent_idx.shape[0] != B:
         raise ValueError("parent_off must be [B,N+1] and parent_idx [B,cap]")
     st = lib().spiffy_accept_walk(

@@ -97,4 +97,21 @@ def assert_decision_parity(w, dec, walk, odec, owalk, tol, margin):
     for name in ("accepted_node", "n_accepted", "path", "next_block"):
         got = getattr(walk, name).cpu().numpy()
         assert np.array_equal(got[seq_safe], getattr(owalk, name)[seq_safe]), name
+    # The walk is integer work: whatever the margins, it must equal the oracle's
+    # walk run on the GPU's own per-node decisions, for every sequence.
+    assert_walk_follows_decisions(w, dec, walk)
     return int(seq_safe.sum())
+
+
+def assert_walk_follows_decisions(w, dec, walk):
+    """The GPU's walk against the oracle's walk on the GPU's own (top_tok,
+    unmask_bits): bit-exact for every sequence."""
+    cfg = w.cfg
+    top = dec.top_tok.cpu().numpy()
+    bits = bits_np(dec.unmask_bits)
+    sel = (bits[..., None] >> np.arange(cfg.block_len, dtype=np.uint64)) & np.uint64(1)
+    nxt = np.where(sel.astype(bool), top, w.block_tokens).astype(np.int32)
+    ow = oracle.accept_walk(w.block_tokens, w.parent_off, w.parent_idx, nxt, bits)
+    for name in ("accepted_node", "n_accepted", "path", "next_block"):
+        assert np.array_equal(getattr(walk, name).cpu().numpy(), getattr(ow, name)), name
+    return ow

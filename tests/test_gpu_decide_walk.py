@@ -27,13 +27,14 @@ def both(logits, tokens, off, idx, mask_id, rule, top_s=1, tau=0.9):
     return dec2, walk2
 
 
-def random_case(seed, B, N, L, V, p_accept=0.7):
+def random_case(seed, B, N, L, V, p_accept=0.7, dtype="f32"):
     """Random logits and a chain-like graph: node m is, with probability
     p_accept, the next state of an earlier node, else a corrupted copy."""
     r = np.random.default_rng(seed)
     mask = V - 1
-    logits = (r.standard_normal((B, N, L, V)) * 3).astype(np.float32)
+    logits = r.standard_normal((B, N, L, V), dtype=np.float32) * np.float32(3)
     logits[..., mask] = -30.0
+    logits = W.round_to(logits, dtype)
     tokens = np.empty((B, N, L), dtype=np.int32)
     lists = []
     for b in range(B):
@@ -194,6 +195,27 @@ def test_lazy_chain_evaluation_equals_the_eager_call_on_the_path(B, N, L, V):
         assert on_path[:, 0].all()
     if N > 2:
         assert hops > 0
+
+
+@pytest.mark.parametrize("B,N,L,V,dtype", [(64, 8, 32, 1000, "f32"), (33, 16, 4, 70000, "bf16"),
+                                           (7, 12, 64, 9000, "f32"), (40, 5, 32, 20000, "bf16")])
+def test_lazy_call_with_more_items_than_resident_thread_blocks(B, N, L, V, dtype):
+    """B * L * slices exceeds what the device holds at once (six thread blocks
+    per SM): every block then takes several (position, slice) items per level,
+    each waiting on another sequence's epoch."""
+    per_slice = 8192 if dtype == "bf16" else 4096
+    items = B * L * -(-V // per_slice)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert items > 6 * sms
+    logits, tokens, off, idx, mask = random_case(B * 1000 + N, B, N, L, V, p_accept=0.9, dtype=dtype)
+    hops = 0
+    for rule, S, tau in ((spiffy.RULE_TOPS, 1, 0.0), (spiffy.RULE_THRESHOLD, 1, 0.5)):
+        for _ in range(3):  # the interleaving of the blocks differs from run to run, the bits must not
+            walk, lwalk, on_path = lazy_vs_eager(logits, tokens, off, idx, mask, rule, S, tau,
+                                                 dtype=torch.bfloat16 if dtype == "bf16" else None)
+            assert int(lwalk.dev_status.sum()) == 0
+        hops += int(walk.n_accepted.sum())
+    assert hops > B  # deep walks: several levels per sequence
 
 
 def test_lazy_chain_evaluation_at_the_benchmark_shapes():

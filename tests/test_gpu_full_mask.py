@@ -54,3 +54,27 @@ def test_blocks_longer_than_a_key_tile(B, N, L, P, Hq, Hkv):
     assert np.abs(out.float().cpu().numpy() - want).max() <= G.TOL["bf16"]
     with pytest.raises(spiffy.SpiffyError):
         spiffy.spiffy_graph_attention(dev(q), dev(kp), dev(vp), dev(kb), dev(vb), kernel=spiffy.ATTN_SIMT)
+
+
+@pytest.mark.parametrize("B,N,L,n_blocks,k,Hq,Hkv", [(1, 4, 32, 8, 5, 32, 32), (2, 8, 32, 6, 3, 8, 2),
+                                                     (1, 3, 16, 4, 0, 4, 4), (1, 16, 32, 20, 19, 28, 4)])
+def test_blockwise_causal_context(B, N, L, n_blocks, k, Hq, Hkv):
+    """Block-causal models (last sentence of the caption of Fig. 3; App. A.2):
+    the packed call for block k takes the cache of the blocks before it as its
+    context -- a view of the sequence's cache, no copy -- and must equal the
+    oracle that masks the whole sequence block-causally."""
+    r = np.random.default_rng(n_blocks * 10 + k)
+    d = 128
+    T = n_blocks * L
+    k_seq, v_seq = bf16(r, B, T, Hkv, d), bf16(r, B, T, Hkv, d)
+    q, kb, vb = bf16(r, B, N, L, Hq, d), bf16(r, B, N, L, Hkv, d), bf16(r, B, N, L, Hkv, d)
+    ks_dev, vs_dev = k_seq.cuda(), v_seq.cuda()
+    if B == 1 and k > 0:  # a prefix of the cache is contiguous: pass the view itself
+        kp, vp = ks_dev[:, :k * L], vs_dev[:, :k * L]
+    else:
+        kp, vp = (ks_dev[:, :k * L].contiguous(), vs_dev[:, :k * L].contiguous()) if k else (None, None)
+    out = spiffy.spiffy_graph_attention(q.cuda(), kp, vp, kb.cuda(), vb.cuda(), kernel=spiffy.ATTN_TCGEN05)
+    torch.cuda.synchronize()
+    f = lambda t: t.float().numpy()
+    want = full_mask.blockwise_causal_attention(f(q), f(k_seq), f(v_seq), f(kb), f(vb), k)
+    assert np.abs(out.float().cpu().numpy() - want).max() <= G.TOL["bf16"]

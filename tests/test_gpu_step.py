@@ -15,12 +15,23 @@ import gpu_util as G
 pytestmark = pytest.mark.gpu
 
 
+_full_size = {}
+
+
+def long_batched_workload():
+    """Configuration 4's decision inputs (2 GB on the host), drawn once."""
+    if "w" not in _full_size:
+        cfg = W.config(4)
+        _full_size["w"] = W.make(cfg, W.seed_for(4, 0), attention=False)
+    return _full_size["w"]
+
+
 def test_full_size_long_batched_decision_sampled():
     """Configuration 4 at full size: 4 x 32 x 32 rows of 126464 logits.  The
     oracle evaluates a sample of nodes; the walk is then checked by running
     the oracle's walk on the GPU's own per-node decisions (integer work)."""
     cfg = W.config(4)
-    w = W.make(cfg, W.seed_for(4, 0), attention=False)
+    w = long_batched_workload()
     dec, walk = G.gpu_decide(w)
     conf = dec.conf.cpu().numpy()
     top = dec.top_tok.cpu().numpy()
@@ -44,6 +55,27 @@ def test_full_size_long_batched_decision_sampled():
     for name in ("accepted_node", "n_accepted", "path", "next_block"):
         assert np.array_equal(getattr(walk, name).cpu().numpy(), getattr(ow, name)), name
     assert ow.n_accepted.max() >= 1
+
+
+def test_full_size_long_batched_lazy_call_equals_the_eager_one():
+    """Configuration 4 at full size through spiffy_decide_walk_lazy: 4 x 32 x 16
+    (position, slice) items, more than the device holds thread blocks, so every
+    block loops over items of several sequences.  Walk outputs and the on-path
+    decisions must be the eager call's bits; the walk itself is checked with the
+    oracle's walk on the eager call's per-node decisions."""
+    import test_gpu_decide_walk as T
+    cfg = W.config(4)
+    w = long_batched_workload()
+    for _ in range(2):
+        walk, lwalk, on_path = T.lazy_vs_eager(w.logits, w.block_tokens, w.parent_off, w.parent_idx,
+                                               cfg.mask_id, cfg.rule, cfg.top_s, cfg.threshold,
+                                               dtype=torch.bfloat16)
+        assert int(lwalk.dev_status.sum()) == 0
+    lg, tk = G.to_dev(w.logits, torch.bfloat16), G.to_dev(w.block_tokens)
+    dec = spiffy.spiffy_unmask_decide(lg, tk, cfg.mask_id, cfg.rule, cfg.top_s, cfg.threshold)
+    ow = G.assert_walk_follows_decisions(w, dec, lwalk)
+    assert ow.n_accepted.max() >= 1 and on_path.sum() > cfg.batch
+    _full_size.clear()  # 2 GB of host memory
 
 
 def gpu_backends(dtype=torch.float32, kernel=spiffy.ATTN_AUTO):

@@ -51,3 +51,39 @@ def test_drafts_do_not_see_the_true_block_and_the_true_rows_see_no_draft():
     nodes3, suffix3 = full_mask.full_sequence_attention(**c3)
     np.testing.assert_allclose(nodes3[:, 0], nodes[:, 0], atol=1e-12)
     np.testing.assert_allclose(suffix3, suffix, atol=1e-12)
+
+
+def test_blockwise_causal_rows_equal_library_attention_on_the_sequence_with_that_node_in_place():
+    """Block-causal models (last sentence of the caption of Fig. 3; App. A.2):
+    what a node gets in the packed call is what its block would get if it stood
+    in the sequence in place of the block being decoded and the model ran with
+    its ordinary block-causal mask -- computed here by torch's attention."""
+    r = np.random.default_rng(9)
+    B, N, L, Hq, Hkv, d, n_blocks, k = 2, 3, 4, 4, 2, 8, 5, 2
+    f = lambda *s: r.standard_normal(s).astype(np.float32).astype(np.float64)
+    T = n_blocks * L
+    q_seq, k_seq, v_seq = f(B, T, Hq, d), f(B, T, Hkv, d), f(B, T, Hkv, d)
+    q_nodes, k_block, v_block = f(B, N, L, Hq, d), f(B, N, L, Hkv, d), f(B, N, L, Hkv, d)
+    got = full_mask.blockwise_causal_attention(q_nodes, k_seq, v_seq, k_block, v_block, k)
+    blk = np.arange(T) // L
+    causal = torch.from_numpy(blk[:, None] >= blk[None, :])  # row block >= key block
+    t = lambda a: torch.from_numpy(a).permute(0, 2, 1, 3)
+    for n in range(N):
+        qs, ks, vs = q_seq.copy(), k_seq.copy(), v_seq.copy()
+        qs[:, k * L:(k + 1) * L] = q_nodes[:, n]
+        ks[:, k * L:(k + 1) * L] = k_block[:, n]
+        vs[:, k * L:(k + 1) * L] = v_block[:, n]
+        rep = Hq // Hkv
+        want = torch.nn.functional.scaled_dot_product_attention(
+            t(qs), t(ks).repeat_interleave(rep, 1), t(vs).repeat_interleave(rep, 1), attn_mask=causal)
+        want = want.permute(0, 2, 1, 3).numpy()[:, k * L:(k + 1) * L]
+        np.testing.assert_allclose(got[:, n], want, atol=1e-12)
+    # later blocks are invisible: changing them changes nothing
+    k2, v2 = k_seq.copy(), v_seq.copy()
+    k2[:, k * L:] += 5.0
+    v2[:, k * L:] -= 5.0
+    np.testing.assert_allclose(full_mask.blockwise_causal_attention(q_nodes, k2, v2, k_block, v_block, k), got,
+                               atol=1e-12)
+    # and it is the packed-attention oracle with the earlier blocks as context
+    want = oracle.graph_attention(q_nodes, k_seq[:, :k * L], v_seq[:, :k * L], k_block, v_block)
+    np.testing.assert_allclose(got, want, atol=1e-12)

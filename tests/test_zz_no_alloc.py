@@ -34,9 +34,10 @@ def assert_same(a, b, tokens, mask_id):
     masked = (tokens == mask_id)
     ca, cb = a.conf.cpu().numpy(), b.conf.cpu().numpy()
     assert np.all(np.isneginf(ca[~masked])) and np.all(np.isneginf(cb[~masked]))
-    # same kernels, same fixed merge order: the tolerance of the parity tests is
-    # the bar, equality is what is expected
+    # same reduction, same fixed merge order: the confidences agree bit for bit
+    # (which is well inside the tolerance of the parity tests)
     assert np.max(np.abs(ca[masked] - cb[masked]), initial=0.0) <= G.TOL["bf16"]
+    assert torch.equal(a.conf.view(torch.int32), b.conf.view(torch.int32))
     assert torch.equal(a.top_tok, b.top_tok)
     assert torch.equal(a.unmask_bits, b.unmask_bits)
     assert torch.equal(a.n_unmask, b.n_unmask)
@@ -67,6 +68,25 @@ def test_small_fp32_shape_then_repeat():
                                                  empty_decision(cfg.batch, cfg.n_nodes, cfg.block_len), cfg.top_s)
         torch.cuda.synchronize()
         assert_same(got, want, w.block_tokens, cfg.mask_id)
+
+
+def test_the_call_allocates_no_device_memory():
+    """What the entry point promises its callers: after the first call on the
+    device (which looks up the array's address), a call changes neither the
+    driver's free-memory figure nor torch's allocation counters."""
+    cfg = W.config(1)
+    w = W.make(cfg, W.seed_for(1, 4), attention=False)
+    logits, tokens = G.to_dev(w.logits), G.to_dev(w.block_tokens)
+    out = empty_decision(cfg.batch, cfg.n_nodes, cfg.block_len)
+    spiffy.spiffy_unmask_decide_static(logits, tokens, cfg.mask_id, cfg.rule, out, cfg.top_s)
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    count0 = torch.cuda.memory_stats()["allocation.all.allocated"]
+    for _ in range(3):
+        spiffy.spiffy_unmask_decide_static(logits, tokens, cfg.mask_id, cfg.rule, out, cfg.top_s)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    assert torch.cuda.memory_stats()["allocation.all.allocated"] == count0
 
 
 def test_shapes_beyond_the_fixed_scratch_are_refused():
