@@ -15,9 +15,14 @@ acceptance walk (step 5).  The metric is verify steps per second.
             VerifyStep.run_host (host-to-device copies of everything the step
             reads -- of the logits, the rows of still-masked positions -- and
             the device-to-host read of the verdict inside the timed region).
-`roofline`: the dominant kernel (the decision reduce) against the measured HBM
-            copy bandwidth; its duration comes from a second pass that replays
-            the decision call alone over the same rotation of input sets.
+`roofline`: the kernel with the largest share of a step (the attention kernel)
+            against the roof that binds it at this shape, timed alone by
+            replaying its call over the same rotation of input sets; the
+            decision kernel likewise under `roofline_decision`.
+`composite_model_step`: a step as a whole model runs it, one attention call
+            per layer on distinct q/K/V, then one decision + walk.
+`other_shapes`: the attention and decision calls at the configurations where
+            the tensor and HBM rooflines bind.
 `cpu_baseline` / `--impl reference`: the CPU oracle as it stands, timed on the
             host cores (a reported baseline, not a target).
 
@@ -41,9 +46,6 @@ METRIC = "draft-graph verify steps/sec at LLaDA-8B shape"
 UNIT = "steps/s"
 WORKLOAD = "config2-llada8b: B=1 N=8 L=32 P=512 Hq=Hkv=32 d=128 bf16, V=126464, threshold 0.9"
 N_SETS = 6  # rotating input sets; 6 x 79.4 MB = 477 MB > 126 MB of L2
-# dram__bytes_read.sum + dram__bytes_write.sum of one decide_reduce_kernel launch at this workload
-# (ncu capture summarised under profiles/); set to None whenever that kernel changes
-NCU_REDUCE_TRAFFIC_BYTES = 41.77e6
 
 
 def parse():
@@ -56,6 +58,8 @@ def parse():
     ap.add_argument("--nodes", type=int, default=None, help="node count for configuration 5")
     ap.add_argument("--attn-kernel", default="auto", choices=["auto", "simt", "tcgen05"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-composite", action="store_true", help="skip the whole-model (one attention call per layer) step")
+    ap.add_argument("--no-other-shapes", action="store_true", help="skip the timing of the other configurations")
     ap.add_argument("--part", default="step", choices=["step", "attention", "decide", "decide_walk", "decide_walk_lazy", "decide_sampled", "lmhead", "draft"],
                     help="time one library call alone on any configuration (for profiling); "
                          "the benchmark line itself is --part step")
@@ -390,6 +394,154 @@ def run_draft_part(args, cfg):
                       "input_sets": n_sets, "peaks": peaks["source"], "dev_status": int(out.dev_status.max())}))
 
 
+def kernel_sources_digest(files):
+    """sha256 over the named kernel sources: ties a stored ncu figure to the code it was taken from."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in files:
+        with open(os.path.join(ROOT, "paper_2509_18085_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(key):
+    """DRAM bytes per launch of a kernel as ncu counted them (profiles/ncu_traffic.json, written
+    next to the summary the figure comes from).  None when there is no record or the kernel's
+    sources have changed since the capture."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    try:
+        with open(path) as f:
+            rec = json.load(f)[key]
+        if rec["sources_sha256_16"] != kernel_sources_digest(rec["sources"]):
+            return None, f"stale: {rec['sources']} changed since the capture in {rec['summary']}"
+        return float(rec["dram_bytes_per_launch"]), f"ncu dram read+write bytes per launch, {rec['summary']}"
+    except (OSError, KeyError, ValueError):
+        return None, "no ncu record"
+
+
+class GraphTimer:
+    """Times CUDA graphs on one stream with CUDA events: every measurement is the
+    median of `repeats` regions, each region replaying the graph until at least
+    `min_region_s` of device time has passed."""
+
+    def __init__(self, stream, repeats=5, min_region_s=0.04):
+        import torch
+        self.torch = torch
+        self.stream = stream
+        self.repeats = repeats
+        self.min_region_s = min_region_s
+
+    def capture(self, fns):
+        torch = self.torch
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=self.stream):
+            for fn in fns:
+                fn()
+        return g
+
+    def region(self, graph, replays):
+        torch = self.torch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(self.stream)
+        for _ in range(replays):
+            graph.replay()
+        e1.record(self.stream)
+        self.stream.synchronize()
+        return e0.elapsed_time(e1) * 1e-3
+
+    def measure(self, graph, min_replays=1, warm_replays=3):
+        """(seconds per replay: median over the regions, replays per region, all regions' values)."""
+        for _ in range(max(1, warm_replays)):
+            graph.replay()
+        self.stream.synchronize()
+        replays = max(1, min_replays)
+        t = self.region(graph, replays)
+        while t < self.min_region_s and replays < (1 << 20):  # grow the region to the minimum length
+            replays = max(replays + 1, int(replays * min(8.0, 1.3 * self.min_region_s / max(t, 1e-7))))
+            t = self.region(graph, replays)
+        per = [self.region(graph, replays) / replays for _ in range(self.repeats)]
+        return statistics.median(per), replays, per
+
+
+def device_attention_inputs(cfg, n_sets, seed):
+    """Random q/k/v of the configuration's shapes drawn on the device (N(0,1), bf16): input
+    data for timing the shapes whose parity the tests cover."""
+    import torch
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    B, N, L, P = cfg.batch, cfg.n_nodes, cfg.block_len, cfg.prefix_len
+    r = lambda *shape: torch.randn(shape, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    return [(r(B, N, L, cfg.n_q_heads, cfg.head_dim), r(B, P, cfg.n_kv_heads, cfg.head_dim),
+             r(B, P, cfg.n_kv_heads, cfg.head_dim), r(B, N, L, cfg.n_kv_heads, cfg.head_dim),
+             r(B, N, L, cfg.n_kv_heads, cfg.head_dim)) for _ in range(n_sets)]
+
+
+def other_shapes(timer, peaks):
+    """The attention call where the tensor roofline binds (configurations 3, 4, 5 with 64
+    nodes) and the decision call where HBM binds (3, 4), each alone on L2-cold inputs."""
+    import torch
+    from paper_2509_18085_b200 import spiffy
+    from paper_2509_18085_b200 import workloads as W
+    out = {"attention": {}, "decision": {}}
+    for index, nodes in ((3, None), (4, None), (5, 64)):
+        cfg = W.config(index, nodes)
+        attn_bytes, _, flops = algorithmic_bytes(cfg, 0)
+        n_sets = max(1, min(16, int(300e6 // attn_bytes) + 1))
+        sets = device_attention_inputs(cfg, n_sets, 40 + index)
+        outs = torch.empty_like(sets[0][0])
+        desc = spiffy.attn_desc(sets[0][0], sets[0][1], sets[0][3], 0.0, spiffy.ATTN_TCGEN05)
+        ws = torch.empty(max(16, spiffy.spiffy_graph_attention_workspace(desc)), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        fns = [lambda x=x: spiffy.spiffy_graph_attention(*x, out=outs, kernel=spiffy.ATTN_TCGEN05,
+                                                         dev_status=status, workspace=ws) for x in sets]
+        for fn in fns:
+            fn()
+        timer.stream.synchronize()
+        sec, replays, _ = timer.measure(timer.capture(fns))
+        sec /= n_sets
+        tf = flops / sec / 1e12
+        name = f"config{index}" + (f"-N{nodes}" if nodes else "")
+        out["attention"][name] = {
+            "us_per_call": sec * 1e6, "tflops": tf, "frac_of_bf16_burst_peak": tf / peaks["bf16_tflops"],
+            "frac_of_bf16_sustained_peak": tf / peaks["bf16_tflops_sustained"],
+            "gbs": attn_bytes / sec / 1e9, "frac_of_hbm": attn_bytes / sec / 1e9 / peaks["hbm_gbs"],
+            "input_sets": n_sets, "calls_timed": replays * n_sets * timer.repeats, "dev_status": int(status)}
+        del sets, outs, ws, fns
+        torch.cuda.empty_cache()
+    for index in (3, 4):
+        cfg = W.config(index)
+        B, N, L, V = cfg.batch, cfg.n_nodes, cfg.block_len, cfg.vocab
+        g = torch.Generator(device="cuda").manual_seed(60 + index)
+        # every sequence's nodes keep about 0.55-0.7 of their positions masked, as the generated graphs do
+        tokens = torch.where(torch.rand((B, N, L), generator=g, device="cuda") < 0.62, cfg.mask_id, 3).to(torch.int32)
+        masked = int((tokens == cfg.mask_id).sum())
+        by = masked * V * 2 + masked * 12
+        n_sets = max(1, min(4, int(300e6 // by) + 1))
+        sets = []
+        for _ in range(n_sets):
+            lg = torch.empty((B, N, L, V), dtype=torch.bfloat16, device="cuda")
+            for b in range(B):  # N(0, 2) drawn sequence by sequence: bounded scratch
+                lg[b] = (torch.randn((N, L, V), generator=g, device="cuda") * 2.0).to(torch.bfloat16)
+            sets.append(lg)
+        dec = None
+        desc = spiffy.decide_desc(sets[0], tokens, cfg.mask_id, cfg.rule, cfg.top_s, cfg.threshold)
+        ws = torch.empty(max(16, spiffy.spiffy_unmask_decide_workspace(desc)), dtype=torch.uint8, device="cuda")
+        dec = spiffy.spiffy_unmask_decide(sets[0], tokens, cfg.mask_id, cfg.rule, cfg.top_s, cfg.threshold, workspace=ws)
+        fns = [lambda lg=lg: spiffy.spiffy_unmask_decide(lg, tokens, cfg.mask_id, cfg.rule, cfg.top_s, cfg.threshold,
+                                                         out=dec, workspace=ws) for lg in sets]
+        timer.stream.synchronize()
+        sec, replays, _ = timer.measure(timer.capture(fns))
+        sec /= n_sets
+        out["decision"][f"config{index}"] = {
+            "us_per_call": sec * 1e6, "gbs": by / sec / 1e9, "frac_of_hbm": by / sec / 1e9 / peaks["hbm_gbs"],
+            "algorithmic_bytes": by, "masked_rows": masked, "input_sets": n_sets,
+            "calls_timed": replays * n_sets * timer.repeats, "dev_status": int(dec.dev_status.max())}
+        del sets, ws, fns, dec
+        torch.cuda.empty_cache()
+    out["inputs"] = ("random tensors of the configurations' shapes and dtypes drawn on the device "
+                     "(timing is value-independent; parity of these shapes is the tests' job)")
+    return out
+
+
 def main():
     args = parse()
     if args.impl == "reference":
@@ -422,74 +574,97 @@ def main():
     masked_rows = float(np.mean([(w.block_tokens == cfg.mask_id).sum() for w in work]))
     attn_bytes, decide_bytes, attn_flops = algorithmic_bytes(cfg, masked_rows)
     set_bytes = sets[0].nbytes()
+    peaks = measured_peaks()
 
     stream = torch.cuda.Stream()
     sampler = ClockSampler(local)
     with torch.cuda.stream(stream):
-        # eager warm-up (also loads the kernels), then capture one rotation
+        timer = GraphTimer(stream)
+        # eager warm-up (also loads the kernels), then capture one rotation over the input sets
         for i in range(max(3, min(args.warmup, 2 * N_SETS))):
             step.run(sets[i % N_SETS])
         stream.synchronize()
         before = spiffy.launch_count()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=stream):
-            for x in sets:
-                step.run(x)
+        graph = timer.capture([lambda x=x: step.run(x) for x in sets])
         launches_per_step = (spiffy.launch_count() - before) / N_SETS
-        replays = max(1, args.steps // N_SETS)
-        steps = replays * N_SETS
-        warm_replays = max(1, -(-args.warmup // N_SETS))
+        # whole rotations only: the asked-for counts are rounded up, never down
+        min_replays = max(1, -(-args.steps // N_SETS))
+        warm_replays = max(1, -(-max(3, args.warmup) // N_SETS))
 
         sampler.start()
-        for _ in range(warm_replays):
-            graph.replay()
-        stream.synchronize()
         replicas.barrier(ranks)
         torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(replays):
-            graph.replay()
-        e1.record(stream)
-        stream.synchronize()
+        sec_replay, replays, regions = timer.measure(graph, min_replays, warm_replays)
         replicas.barrier(ranks)
         torch.cuda.synchronize()
-        ms_total = e0.elapsed_time(e1)
+        steps = replays * N_SETS
+        ms_total = sec_replay * replays * 1e3  # the median region
 
-        # per-call durations: the same rotation, one library call per graph node
+        # each library call alone, over the same rotation of input sets
         def call_seconds(fn):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                for x in sets:
-                    fn(x)
-            reps = max(2, min(replays, 200))
-            g.replay()
-            stream.synchronize()
-            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a0.record(stream)
-            for _ in range(reps):
-                g.replay()
-            a1.record(stream)
-            stream.synchronize()
-            return a0.elapsed_time(a1) * 1e-3 / (reps * N_SETS)
+            before = spiffy.launch_count()
+            g = timer.capture([lambda x=x: fn(x) for x in sets])
+            kernels = (spiffy.launch_count() - before) / N_SETS
+            sec, _, _ = timer.measure(g)
+            return sec / N_SETS, kernels
 
-        t_attn = call_seconds(step.attention)
-        t_dec = call_seconds(step.decide)
-        t_walk = call_seconds(step.accept)
-        t_dw = call_seconds(step.decide_accept)
+        t_attn, k_attn = call_seconds(step.attention)
+        t_dec, k_dec = call_seconds(step.decide)
+        t_walk, _ = call_seconds(step.accept)
+        t_dw, k_dw = call_seconds(step.decide_accept)
+
+        # one verification step of a whole model: the attention runs once per layer, each layer
+        # on its own q/K/V (32 layers x 16.8 MB: L2-cold by construction), then one decision + walk
+        composite = None
+        if args.config in (2, 3, 4, 5) and not args.no_composite:
+            layers = 28 if args.config == 3 else 32
+            layer_sets = device_attention_inputs(cfg, layers, 7)
+            layer_fns = [lambda x=x: spiffy.spiffy_graph_attention(*x, out=step.attn_out, kernel=kernel,
+                                                                   dev_status=step.attn_status,
+                                                                   workspace=step.attn_ws) for x in layer_sets]
+            for fn in layer_fns[:2]:
+                fn()
+            stream.synchronize()
+            before = spiffy.launch_count()
+            cg = timer.capture([fn for fn in layer_fns] + [lambda: step.decide_accept(sets[0]),
+                                                           ] + [fn for fn in layer_fns] +
+                               [lambda: step.decide_accept(sets[1])])
+            launches_c = (spiffy.launch_count() - before) / 2
+            sec_c, replays_c, _ = timer.measure(cg)
+            sec_c /= 2
+            ag = timer.capture(layer_fns)
+            sec_layers, _, _ = timer.measure(ag)
+            composite = {
+                "layers_per_step": layers, "layer_count_source": "public model card, not the paper",
+                "value": 1.0 / sec_c, "unit": UNIT, "ms_per_step": sec_c * 1e3,
+                "attention_us_per_layer": sec_layers / layers * 1e6,
+                "attention_share": sec_layers / sec_c, "gpu_launches_per_step": launches_c,
+                "steps_timed": replays_c * 2 * timer.repeats,
+                "attention_frac_of_binding_roofline":
+                    max(attn_flops / (peaks["bf16_tflops"] * 1e12), attn_bytes / (peaks["hbm_gbs"] * 1e9))
+                    / (sec_layers / layers),
+                "inputs": "per-layer q/K/V drawn on the device, N(0,1) bf16; logits of the step's own sets"}
+            del layer_sets, layer_fns, cg, ag
+
+        shapes = None
+        if rank == 0 and world == 1 and args.config == 2 and not args.no_other_shapes:
+            shapes = other_shapes(timer, peaks)
 
         # end to end from pinned host memory
-        n_e2e = max(3, min(50, steps))
+        n_e2e = max(5, min(50, steps))
         for _ in range(3):
             step.run_host(host0)
         torch.cuda.synchronize()
-        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        h0.record(stream)
-        for _ in range(n_e2e):
-            step.run_host(host0)
-        h1.record(stream)
-        stream.synchronize()
-        ms_e2e = h0.elapsed_time(h1) / n_e2e
+        e2e_regions = []
+        for _ in range(3):
+            h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            h0.record(stream)
+            for _ in range(n_e2e):
+                step.run_host(host0)
+            h1.record(stream)
+            stream.synchronize()
+            e2e_regions.append(h0.elapsed_time(h1) / n_e2e)
+        ms_e2e = statistics.median(e2e_regions)
         clocks = sampler.stop()
         status = int(step.attn_status.item()) | int(step.decision.dev_status.max().item()) | \
             int(step.walk.dev_status.max().item())
@@ -500,25 +675,42 @@ def main():
     value = replicas.whole_job_rate(ranks, steps, ms_total)
     e2e_value = replicas.whole_job_rate(ranks, 1, ms_e2e)
 
-    peaks = measured_peaks()
-    roofline = {
-        "kernel": "decide_reduce_kernel (timed as the spiffy_unmask_decide call: reduce + finalize)",
-        "bound": "hbm", "achieved": decide_bytes / t_dec / 1e9, "peak": peaks["hbm_gbs"],
-        "unit": "GB/s", "frac": decide_bytes / t_dec / 1e9 / peaks["hbm_gbs"],
-        "peak_source": peaks["source"] + " (burst copy)", "traffic": NCU_REDUCE_TRAFFIC_BYTES,
-        "traffic_note": "dram read+write bytes of one decide_reduce_kernel launch, ncu capture in "
-                        "profiles/decide_reduce_kernel_config2.md",
-        "algorithmic_bytes": decide_bytes, "seconds": t_dec,
-    }
+    # rooflines: every kernel against the roof that binds it at this shape
+    t_tensor = attn_flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = attn_bytes / (peaks["hbm_gbs"] * 1e9)
+    attn_bound = "tensor" if t_tensor > t_hbm else "hbm"
     attn_tc = attn_flops / t_attn / 1e12
-    attention = {
-        "seconds": t_attn, "tflops": attn_tc, "frac_of_bf16_peak": attn_tc / peaks["bf16_tflops"],
+    tr_attn, tr_attn_note = ncu_traffic("graph_attention_tc_kernel@config%d" % args.config)
+    attention_roof = {
+        "kernel": "graph_attention_tc_kernel" + (" (+ graph_attention_combine_kernel)" if k_attn > 1 else ""),
+        "timed_as": f"the spiffy_graph_attention call alone ({k_attn:g} kernel(s) per call), graph replay over "
+                    f"{N_SETS} L2-cold input sets, CUDA events on the launching stream",
+        "bound": attn_bound,
+        "achieved": attn_bytes / t_attn / 1e9 if attn_bound == "hbm" else attn_tc,
+        "peak": peaks["hbm_gbs"] if attn_bound == "hbm" else peaks["bf16_tflops"],
+        "unit": "GB/s" if attn_bound == "hbm" else "TFLOP/s",
+        "frac": max(t_tensor, t_hbm) / t_attn,
+        "peak_source": peaks["source"] + (" (burst copy)" if attn_bound == "hbm" else " (burst GEMM)"),
+        "traffic": tr_attn, "traffic_note": tr_attn_note,
+        "seconds": t_attn, "algorithmic_bytes": attn_bytes, "algorithmic_flops": attn_flops,
+        "tflops": attn_tc, "frac_of_bf16_peak": attn_tc / peaks["bf16_tflops"],
         "gbs": attn_bytes / t_attn / 1e9, "frac_of_hbm": attn_bytes / t_attn / 1e9 / peaks["hbm_gbs"],
-        "algorithmic_bytes": attn_bytes, "algorithmic_flops": attn_flops,
-        "binding_roofline_seconds": max(attn_flops / (peaks["bf16_tflops"] * 1e12),
-                                        attn_bytes / (peaks["hbm_gbs"] * 1e9)),
+        "share_of_step": t_attn / (t_attn + t_dw),
     }
-    attention["frac_of_binding_roofline"] = attention["binding_roofline_seconds"] / t_attn
+    tr_dec, tr_dec_note = ncu_traffic("decide_reduce_kernel@config%d" % args.config)
+    decision_roof = {
+        "kernel": "decide_reduce_kernel" + (" + decide_finalize_kernel" if k_dec > 1 else ""),
+        "timed_as": f"the spiffy_unmask_decide call alone ({k_dec:g} kernel(s) per call), same protocol",
+        "bound": "hbm", "achieved": decide_bytes / t_dec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+        "frac": decide_bytes / t_dec / 1e9 / peaks["hbm_gbs"], "peak_source": peaks["source"] + " (burst copy)",
+        "traffic": tr_dec, "traffic_note": tr_dec_note, "seconds": t_dec, "algorithmic_bytes": decide_bytes,
+        "share_of_step": t_dw / (t_attn + t_dw),
+    }
+    dominant_is_attention = (composite is not None) or t_attn >= t_dw
+    roofline = dict(attention_roof if dominant_is_attention else decision_roof)
+    roofline["why_this_kernel"] = (
+        "largest share of a whole-model step (one attention call per layer)" if composite is not None
+        else "largest share of the single-layer step")
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
@@ -528,16 +720,24 @@ def main():
                    "layers_per_step": 1, "multi_gpu": "independent replicas, no collective",
                    "l2": f"rotating {N_SETS} input sets ({N_SETS * set_bytes / 1e6:.0f} MB) > 126 MB L2",
                    "launch": "CUDA graph of one rotation, replayed",
+                   "protocol": f"median of {timer.repeats} regions of {steps} steps each "
+                               f"(asked: --steps {args.steps} --warmup {args.warmup}, rounded up to whole rotations "
+                               f"and to regions of at least {timer.min_region_s * 1e3:.0f} ms)",
                    "attention_kernel": args.attn_kernel, "masked_rows": masked_rows},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": step.h2d_bytes(host0),
                 "d2h_bytes_per_step": step.d2h_bytes(), "ms_per_step": ms_e2e},
         "gpu_launches": int(round(launches_per_step * steps)),
-        "roofline": roofline, "attention": attention,
+        "roofline": roofline, "roofline_attention": attention_roof, "roofline_decision": decision_roof,
         "per_call_us": {"graph_attention": t_attn * 1e6, "unmask_decide": t_dec * 1e6,
                         "accept_walk": t_walk * 1e6, "decide_walk": t_dw * 1e6},
+        "regions_ms_per_step": [r / N_SETS * 1e3 for r in regions],
         "dev_status": status,
     }
+    if composite is not None:
+        line["composite_model_step"] = composite
+    if shapes is not None:
+        line["other_shapes"] = shapes
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         sec, what = oracle_step_time(cfg, work[0], 80)  # about ten seconds of CPU work
