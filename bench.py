@@ -60,6 +60,8 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-composite", action="store_true", help="skip the whole-model (one attention call per layer) step")
     ap.add_argument("--no-other-shapes", action="store_true", help="skip the timing of the other configurations")
+    ap.add_argument("--no-early-dependents", action="store_true",
+                    help="whole-model step without SPIFFY_ATTN_EARLY_DEPENDENTS on the layers' attention calls")
     ap.add_argument("--part", default="step", choices=["step", "attention", "decide", "decide_walk", "decide_walk_lazy", "decide_sampled", "lmhead", "draft"],
                     help="time one library call alone on any configuration (for profiling); "
                          "the benchmark line itself is --part step")
@@ -619,7 +621,9 @@ def main():
         if args.config in (2, 3, 4, 5) and not args.no_composite:
             layers = 28 if args.config == 3 else 32
             layer_sets = device_attention_inputs(cfg, layers, 7)
-            layer_fns = [lambda x=x: spiffy.spiffy_graph_attention(*x, out=step.attn_out, kernel=kernel,
+            # in a layer loop the next kernel may begin its set-up while this one drains
+            layer_kernel = kernel if args.no_early_dependents else kernel | spiffy.ATTN_EARLY_DEPENDENTS
+            layer_fns = [lambda x=x: spiffy.spiffy_graph_attention(*x, out=step.attn_out, kernel=layer_kernel,
                                                                    dev_status=step.attn_status,
                                                                    workspace=step.attn_ws) for x in layer_sets]
             for fn in layer_fns[:2]:
@@ -643,6 +647,7 @@ def main():
                 "attention_frac_of_binding_roofline":
                     max(attn_flops / (peaks["bf16_tflops"] * 1e12), attn_bytes / (peaks["hbm_gbs"] * 1e9))
                     / (sec_layers / layers),
+                "early_dependents": not args.no_early_dependents,
                 "inputs": "per-layer q/K/V drawn on the device, N(0,1) bf16; logits of the step's own sets"}
             del layer_sets, layer_fns, cg, ag
 

@@ -93,6 +93,13 @@ typedef enum { SPIFFY_RULE_TOPS = 0, SPIFFY_RULE_THRESHOLD = 1 } spiffy_rule;
 #define SPIFFY_ATTN_AUTO 0   /* tensor-core kernel when the shape allows it   */
 #define SPIFFY_ATTN_SIMT 1   /* fp32 CUDA-core kernel (any supported shape)   */
 #define SPIFFY_ATTN_TCGEN05 2 /* tcgen05/TMEM kernel or SPIFFY_EUNSUPPORTED   */
+/* Flag, OR-ed into spiffy_attn_desc.kernel: the next kernel of the stream may be
+ * scheduled while this call's kernel still runs (it is launched as soon as every
+ * thread block of this kernel has started; kernels that order themselves with
+ * cudaGridDependencySynchronize(), as all kernels of this library do, still see
+ * this call's complete output).  For the layer loop of a model, where the next
+ * kernel's set-up then overlaps this kernel's tail.  Tensor-core kernel only. */
+#define SPIFFY_ATTN_EARLY_DEPENDENTS 0x100
 
 /* ------------------------------------------------------------------------- */
 /* Packed draft-graph attention (Sec. 4.3; mask semantics: caption of Fig. 3) */
@@ -108,7 +115,7 @@ typedef struct {
   int32_t head_dim;   /* d in {64, 128}                                      */
   int32_t dtype;      /* spiffy_dtype of q, k, v and out                     */
   float scale;        /* softmax scale; 0 means 1/sqrt(d)                    */
-  int32_t kernel;     /* SPIFFY_ATTN_*                                       */
+  int32_t kernel;     /* SPIFFY_ATTN_AUTO/SIMT/TCGEN05, | SPIFFY_ATTN_EARLY_DEPENDENTS */
 } spiffy_attn_desc;
 
 /* Bytes of scratch spiffy_graph_attention needs for this shape (may be 0). */

@@ -29,7 +29,8 @@ spiffy_status check_attn_desc(const spiffy_attn_desc* d) {
   if (d->n_q_heads % d->n_kv_heads != 0) return SPIFFY_EINVAL;
   if (d->dtype != SPIFFY_F32 && d->dtype != SPIFFY_BF16) return SPIFFY_EINVAL;
   if (!(d->scale >= 0.f) || !(d->scale < INFINITY)) return SPIFFY_EINVAL;
-  if (d->kernel < SPIFFY_ATTN_AUTO || d->kernel > SPIFFY_ATTN_TCGEN05) return SPIFFY_EINVAL;
+  if (d->kernel & ~(0xff | SPIFFY_ATTN_EARLY_DEPENDENTS)) return SPIFFY_EINVAL;
+  if ((d->kernel & 0xff) > SPIFFY_ATTN_TCGEN05) return SPIFFY_EINVAL;
   if (d->block_len > 1024) return SPIFFY_EUNSUPPORTED;
   if (d->head_dim != 64 && d->head_dim != 128) return SPIFFY_EUNSUPPORTED;
   if (d->n_nodes > 65535 || d->batch > 65535) return SPIFFY_EUNSUPPORTED;
@@ -37,7 +38,7 @@ spiffy_status check_attn_desc(const spiffy_attn_desc* d) {
 }
 
 bool use_tc(const spiffy_attn_desc& d) {
-  if (d.kernel == SPIFFY_ATTN_SIMT) return false;
+  if ((d.kernel & 0xff) == SPIFFY_ATTN_SIMT) return false;
   return attention_tc_supported(d);
 }
 
@@ -105,7 +106,7 @@ spiffy_status spiffy_graph_attention(const spiffy_attn_desc* desc, const void* q
     return launch_attention_tc(d, q, k_prefix, v_prefix, k_block, v_block, out,
                                dev_status, workspace, stream);
   }
-  if (d.kernel == SPIFFY_ATTN_TCGEN05) return SPIFFY_EUNSUPPORTED;
+  if ((d.kernel & 0xff) == SPIFFY_ATTN_TCGEN05) return SPIFFY_EUNSUPPORTED;
   if (d.block_len > 64) return SPIFFY_EUNSUPPORTED;  // the CUDA-core kernel keeps a block's rows in registers
   return launch_attention_simt(d, q, k_prefix, v_prefix, k_block, v_block, out, stream);
 }

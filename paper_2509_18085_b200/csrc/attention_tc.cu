@@ -15,24 +15,25 @@
 //
 // Pipeline inside a CTA (320 threads):
 //   warp 0      TMA producer: Q once, then K and V tiles into two rings (seven
-//               32 KB tiles of shared memory in all)
+//               32 KB tiles of shared memory in all); its first loads go out
+//               before the rest of the CTA has finished setting up
 //   warp 1      allocates tensor memory; one lane issues tcgen05.mma:
 //               S = Q K^T (fp32 in TMEM, double buffered), O += P V
-//   warps 2-9   two softmax warpgroups, each with its own S buffer, accumulator
-//               O and running (maximum, sum), so that the exponentials of one
-//               tile overlap the other tile's products: with one M-tile per
-//               CTA the first takes the even key tiles and the second the odd
-//               ones (a CTA with few key tiles leaves it all to the first);
-//               with two M-tiles each warpgroup owns one.  One thread per row
-//               reads S from TMEM, writes P (bf16) back over it as the A
-//               operand of the second product, and rescales its O only when
-//               the maximum grew by more than 2^8 (exact: O and the sum always
-//               share one reference maximum).  At the end the accumulators
-//               are merged where two belong to the same rows, normalised and
-//               stored.
-// With several splits (grid.z) each CTA handles a slice of the key tiles and
-// stores an unnormalised partial (O, reference maximum, sum); a second kernel
-// merges the partials.
+//   warps 2-9   two softmax warpgroups, one thread per row each.  With one
+//               M-tile per CTA they split every key tile by columns (keys
+//               0-63 and 64-127 of the tile), each with its own running
+//               (maximum, sum) and accumulator O, merged once at the end; with
+//               two M-tiles each warpgroup owns one.  A thread reads its scores
+//               from TMEM, writes P (bf16) back over them as the A operand of
+//               the second product, and rescales its O only when the maximum
+//               grew by more than 2^8 (exact: O and the sum always share one
+//               reference maximum).  32-column chunks of a block-key tile that
+//               no row of a warp may see are skipped.
+// With several splits (grid.z) each CTA handles a slice of the key tiles: two
+// slices are the two CTAs of a cluster, which exchange their partials through
+// each other's shared memory and finish half of the output columns each; more
+// slices store unnormalised partials (O, reference maximum, sum) that a second
+// kernel merges.
 //
 // Every wait is bounded; a wait that gives up raises SPIFFY_DEV_TIMEOUT in the
 // caller's status word and the CTA winds down without touching its output.
@@ -59,7 +60,8 @@ constexpr uint32_t kTmemCols = 512;
 // O: 2 x 128 columns, one accumulator per softmax warpgroup
 constexpr uint32_t kColS = 0, kColO = 256;
 constexpr float kRescaleLog2 = 8.0f;
-constexpr int kSoloTiles = 6;  // up to this many key tiles one softmax warpgroup works alone
+// bytes a CTA of a pair receives from its peer: 128 rows x 64 columns of partial O, and (max, sum) per row
+constexpr uint32_t kXchgBytes = BM * 64 * 4 + BM * 8;
 
 // NQ M-tiles per CTA: NQ Q tiles, a K ring of 3 stages and a V ring of 4 - NQ
 // stages: 7 tiles of 32 KB either way.
@@ -70,7 +72,7 @@ struct Smem {
   static constexpr int k = q + NQ * kTileBytes;
   static constexpr int v = k + ks * kTileBytes;
   static constexpr int bars = v + vs * kTileBytes;
-  static constexpr int n_bars = 1 + 4 * kMaxStages + 2 + 2 + 2;
+  static constexpr int n_bars = 1 + 4 * kMaxStages + 2 + 2 + 2 + 2;
   static constexpr int tmem = bars + 8 * n_bars;
   static constexpr int abort_flag = tmem + 8;
   static constexpr int total = abort_flag + 8;
@@ -92,6 +94,7 @@ struct Params {
   float* part_ml;  // [splits][B*Hkv][MT][128][2]
   int32_t* status;
   uint32_t spin_limit;  // polls of one mbarrier wait
+  int early_trigger;    // let the next kernel of the stream begin its set-up while this one runs
 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -100,16 +103,91 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// One thread's NC scores of a row (raw bits in s, -inf where masked): the
+// maximum over the 32-column chunks flagged in `need`.
+template <int NC>
+__device__ __forceinline__ float row_max(const uint32_t (&s)[NC], uint32_t need) {
+  float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+  for (int h = 0; h < NC / 32; ++h) {
+    if ((need >> h) & 1u) {
+#pragma unroll
+      for (int c = 32 * h; c < 32 * h + 32; c += 8) {
+        mx0 = max3(mx0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+        mx1 = max3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+        mx2 = max3(mx2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
+        mx3 = max3(mx3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
+      }
+    }
+  }
+  return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+}
+
+// p = 2^(s * k2 - m_use) for the flagged chunks (zero elsewhere), packed as bf16
+// pairs into pk; returns the sum of the p's (fp32, before rounding to bf16).
+template <int NC>
+__device__ __forceinline__ float row_exps(const uint32_t (&s)[NC], uint32_t need, float k2, float m_use,
+                                          uint32_t (&pk)[NC / 2]) {
+  const uint64_t k22 = pack2(k2, k2), nm2 = pack2(-m_use, -m_use);
+  uint64_t sum_a = pack2(0.f, 0.f), sum_b = pack2(0.f, 0.f);
+#pragma unroll
+  for (int h = 0; h < NC / 32; ++h) {
+    if ((need >> h) & 1u) {
+#pragma unroll
+      for (int c = 32 * h; c < 32 * h + 32; c += 2) {
+        const uint64_t x2 = fma2(pack2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), k22, nm2);
+        float x0, x1;
+        unpack2(x2, x0, x1);
+        const float p0 = ex2(x0), p1 = ex2(x1);
+        if ((c >> 1) & 1) sum_b = add2(sum_b, pack2(p0, p1)); else sum_a = add2(sum_a, pack2(p0, p1));
+        pk[c >> 1] = pack_bf16(p0, p1);
+      }
+    } else {
+#pragma unroll
+      for (int c = 16 * h; c < 16 * h + 16; ++c) pk[c] = 0u;
+    }
+  }
+  float a0, a1;
+  unpack2(add2(sum_a, sum_b), a0, a1);
+  return a0 + a1;
+}
+
 // Bounded wait that ignores the abort flag (used while winding down).
 __device__ __forceinline__ void mbar_wait_quiet(uint64_t* bar, uint32_t parity) {
   for (uint32_t i = 0; i < kSpinLimit; ++i)
     if (mbar_try_wait(bar, parity)) return;
 }
 
-// NQ = 1: the CTA owns one M-tile and its two softmax warpgroups alternate over
-// the key tiles.  NQ = 2: the CTA owns two neighbouring M-tiles, one per
-// warpgroup, and every K/V tile brought into shared memory serves both, which
-// halves the L2-to-SM traffic per flop.
+// Row r of an M-tile sees the columns [lo, hi) of key tile t (tile-relative).
+struct Window {
+  int lo, hi;
+};
+__device__ __forceinline__ Window visible_window(const Params& p, int t, int kb_start, int node) {
+  Window w;
+  if (t < p.TP) {  // context: every row sees every key that exists
+    w.lo = 0;
+    w.hi = min(BN, p.P - t * BN);
+  } else {  // block keys: the row's own node only
+    w.lo = node * p.L - (kb_start + (t - p.TP) * BN);
+    w.hi = w.lo + p.L;
+  }
+  return w;
+}
+
+// NQ = 1: the CTA owns one M-tile.  Its two softmax warpgroups split every key
+// tile by columns: warpgroup w owns the scores of keys 64 w .. 64 w + 63 of the
+// tile, keeps its own running (maximum, sum) and its own accumulator O_w, so
+// that the two never exchange anything per tile and both work on every tile;
+// O_0 and O_1 are merged once, at the end.
+// NQ = 2: the CTA owns two neighbouring M-tiles, one per warpgroup, and every
+// K/V tile brought into shared memory serves both, which halves the L2-to-SM
+// traffic per flop.
 template <int NQ>
 __global__ void __launch_bounds__(kThreads, 1)
 graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
@@ -133,7 +211,9 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
   uint64_t* v_empty = v_full + VS;
   uint64_t* s_full = v_empty + VS;   // [2]
   uint64_t* p_ready = s_full + 2;    // [2]
-  uint64_t* pv_done = p_ready + 2;   // [2], one per softmax warpgroup
+  uint64_t* pv_done = p_ready + 2;   // [2]: NQ = 2 one per warpgroup; NQ = 1 only the first
+  uint64_t* xchg_ready = pv_done + 2;  // pair: the peer's Q tile and first K stage may be overwritten
+  uint64_t* xchg_full = xchg_ready + 1;  // pair: the peer's partial has arrived here
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + SM::tmem);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SM::abort_flag);
 
@@ -142,6 +222,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
   const int bg = blockIdx.y;
   const int b = bg / p.Hkv, g = bg % p.Hkv;
   const int split = blockIdx.z;
+  const bool pair = NQ == 1 && p.pair != 0;
 
   // this CTA's rows and key tiles
   const int nl0 = mt * p.TNL;
@@ -151,19 +232,72 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
   const int kb_start = n_lo * p.L;
   const int TB = ((n_hi - n_lo + 1) * p.L + BN - 1) / BN;
   const int T_all = p.TP + TB;
-  const int t_begin = (int)((int64_t)split * T_all / p.splits);
-  const int t_end = (int)((int64_t)(split + 1) * T_all / p.splits);
+  const int t_begin = split * T_all / p.splits;  // small numbers: splits <= T_all <= a few thousand
+  const int t_end = (split + 1) * T_all / p.splits;
   const int T = t_end - t_begin;
 
+  // ---- producers.  K tiles (and Q) are loaded by lane 0 of warp 0, V tiles by
+  // lane 0 of warp 1 until that thread turns to issuing the products; each
+  // initialises the barriers of its ring itself, so that its first loads go out
+  // at once, ahead of the rest of the set-up (tensor-memory allocation, the
+  // CTA-wide barrier).  `produce` issues tile j of one ring; may_wait = false:
+  // only if its stage is still in its first round (nothing to wait for).
+  int issued_k = 0, issued_v = 0;
+  bool prod_ok = true;
+  auto produce = [&](bool is_k, int j, bool may_wait) -> bool {
+    const int depth = is_k ? KS : VS;
+    const int stage = j % depth;
+    const uint32_t round = (uint32_t)(j / depth);
+    if (round > 0) {
+      if (!may_wait) return false;
+      if (!mbar_wait((is_k ? k_empty : v_empty) + stage, (round & 1u) ^ 1u, abort_flag, p.spin_limit)) {
+        prod_ok = false;
+        return false;
+      }
+    }
+    uint64_t* full = (is_k ? k_full : v_full) + stage;
+    const int t = t_begin + j;
+    const bool ctx = t < p.TP;
+    const CUtensorMap* m = is_k ? (ctx ? &tm_kp : &tm_kb) : (ctx ? &tm_vp : &tm_vb);
+    const int key0 = ctx ? t * BN : kb_start + (t - p.TP) * BN;
+    uint8_t* dst = (is_k ? sk : sv) + stage * kTileBytes;
+    mbar_arrive_expect_tx(full, kTileBytes);
+    tma_load_4d(dst, m, full, 0, g, key0, b);
+    tma_load_4d(dst + kHalfBytes, m, full, 64, g, key0, b);
+    if (is_k) issued_k = j + 1; else issued_v = j + 1;
+    return true;
+  };
+
   if (threadIdx.x == 0) {
+    prefetch_tensormap(&tm_q);  // the descriptors are kernel parameters
+    prefetch_tensormap(p.TP > 0 ? &tm_kp : &tm_kb);
     mbar_init(q_full, 1);
     for (int i = 0; i < KS; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
-    for (int i = 0; i < VS; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_ready + i, 128); }
+    for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_ready + i, NQ == 1 ? 256 : 128); }
     mbar_init(pv_done, 1);
     mbar_init(pv_done + 1, 1);
+    mbar_init(xchg_ready, 1);
+    mbar_init(xchg_full, 1);
     *abort_flag = 0;
     mbar_fence_init();
+    if (pair) mbar_arrive_expect_tx(xchg_full, kXchgBytes);  // what the peer will send in the epilogue
+    cudaGridDependencySynchronize();
+    if (T > 0) {
+      mbar_arrive_expect_tx(q_full, (uint32_t)NQ * 2u * rows_box * 128u);
+#pragma unroll
+      for (int q = 0; q < NQ; ++q) {  // an M-tile beyond the last one reads as zeros
+        tma_load_4d(sq + q * kTileBytes, &tm_q, q_full, 0, g * p.group, nl0 + q * p.TNL, b);
+        tma_load_4d(sq + q * kTileBytes + kHalfBytes, &tm_q, q_full, 64, g * p.group,
+                    nl0 + q * p.TNL, b);
+      }
+      while (issued_k < T && produce(true, issued_k, false)) {}
+    }
+  } else if (threadIdx.x == 32) {
+    prefetch_tensormap(p.TP > 0 ? &tm_vp : &tm_vb);
+    for (int i = 0; i < VS; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
+    mbar_fence_init();
+    cudaGridDependencySynchronize();
+    while (issued_v < T && produce(false, issued_v, false)) {}
   }
   // rows of the Q tile that the TMA box does not write must be finite
   for (int i = rows_box * 8 + threadIdx.x; i < BM * 8; i += kThreads) {
@@ -177,48 +311,26 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
-  if (threadIdx.x == 0) {  // the descriptors are kernel parameters: fetch them ahead of the wait
-    prefetch_tensormap(&tm_q);
-    prefetch_tensormap(p.TP > 0 ? &tm_kp : &tm_kb);
-    prefetch_tensormap(p.TP > 0 ? &tm_vp : &tm_vb);
-  }
-  // everything above is on-chip set-up; global memory is touched from here on
+  // pair: both CTAs' barriers exist before either touches the other's (waited for in the epilogue)
+  if (pair) cluster_arrive();
+  if (p.early_trigger) pdl_launch_dependents();
+  // everything above is on-chip set-up (thread 0 aside); global memory is touched from here on
   cudaGridDependencySynchronize();
 
   if (warp == 0) {
     // ------------------------------------------------------------ producer --
     if (lane == 0 && T > 0) {
-      mbar_arrive_expect_tx(q_full, (uint32_t)NQ * 2u * rows_box * 128u);
-#pragma unroll
-      for (int q = 0; q < NQ; ++q) {  // an M-tile beyond the last one reads as zeros
-        tma_load_4d(sq + q * kTileBytes, &tm_q, q_full, 0, g * p.group, nl0 + q * p.TNL, b);
-        tma_load_4d(sq + q * kTileBytes + kHalfBytes, &tm_q, q_full, 64, g * p.group,
-                    nl0 + q * p.TNL, b);
+      // the rest of both rings, in the order the products need them: K(j+1) before V(j)
+      issued_v = min(T, VS);             // what warp 1's lane issued before the barrier
+      int jk = issued_k, jv = issued_v;
+      while (prod_ok && (jk < T || jv < T)) {
+        if (jk < T && jk <= jv + 1) {
+          if (produce(true, jk, true)) ++jk;
+        } else if (jv < T) {
+          if (produce(false, jv, true)) ++jv;
+        }
       }
-      int issued_k = 0, issued_v = 0;
-      bool ok = true;
-      auto load = [&](bool is_k, int j) {
-        const int stage = j % (is_k ? KS : VS);
-        const uint32_t round = (uint32_t)(j / (is_k ? KS : VS));
-        uint64_t* empty = (is_k ? k_empty : v_empty) + stage;
-        uint64_t* full = (is_k ? k_full : v_full) + stage;
-        if (!mbar_wait(empty, (round & 1u) ^ 1u, abort_flag, p.spin_limit)) { ok = false; return; }
-        const int t = t_begin + j;
-        const bool ctx = t < p.TP;
-        const CUtensorMap* m = is_k ? (ctx ? &tm_kp : &tm_kb) : (ctx ? &tm_vp : &tm_vb);
-        const int key0 = ctx ? t * BN : kb_start + (t - p.TP) * BN;
-        uint8_t* dst = (is_k ? sk : sv) + stage * kTileBytes;
-        mbar_arrive_expect_tx(full, kTileBytes);
-        tma_load_4d(dst, m, full, 0, g, key0, b);
-        tma_load_4d(dst + kHalfBytes, m, full, 64, g, key0, b);
-        if (is_k) issued_k = j + 1; else issued_v = j + 1;
-      };
-      load(true, 0);
-      for (int j = 0; j < T && ok; ++j) {
-        if (j + 1 < T) load(true, j + 1);
-        if (ok) load(false, j);
-      }
-      if (!ok) {
+      if (!prod_ok) {
         // winding down: let the copies already in flight land before exit
         mbar_wait_quiet(q_full, 0);
         for (int j = max(0, issued_k - KS); j < issued_k; ++j)
@@ -232,31 +344,16 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     if (lane == 0 && T > 0) {
       constexpr uint32_t idesc_s = idesc_bf16_f32(BM, BN, false, false);
       constexpr uint32_t idesc_o = idesc_bf16_f32(BM, HD, false, true);
+      constexpr uint32_t hi = desc_hi_sw128(1024);
+      const uint32_t q_lo = desc_lo_sw128(smem_u32(sq), 16);
+      const uint32_t k_lo = desc_lo_sw128(smem_u32(sk), 16);
+      const uint32_t v_lo = desc_lo_sw128(smem_u32(sv), kHalfBytes);
       bool ok = mbar_wait(q_full, 0, abort_flag, p.spin_limit);
       // S = Q K^T of key tile j into S buffer `buf`, from Q tile `qt`
       auto issue_s = [&](int j, int buf, int qt) {
-        const uint32_t q_addr = smem_u32(sq + qt * kTileBytes);
-        const uint32_t k_addr = smem_u32(sk + (j % KS) * kTileBytes);
-        const uint32_t d = tmem + kColS + (uint32_t)buf * BN;
-#pragma unroll
-        for (int kk = 0; kk < HD / 16; ++kk) {
-          const uint32_t off = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-          umma_ss(d, smem_desc_sw128(q_addr + off, 16, 1024),
-                  smem_desc_sw128(k_addr + off, 16, 1024), idesc_s, kk > 0);
-        }
+        umma_ss_k128(tmem + kColS + (uint32_t)buf * BN, q_lo + (uint32_t)qt * (kTileBytes >> 4),
+                     k_lo + (uint32_t)(j % KS) * (kTileBytes >> 4), hi, idesc_s, 0u);
         umma_commit(s_full + buf);
-      };
-      // O[buf] (+)= P[buf] V of key tile j; `first` starts the accumulator
-      auto issue_pv = [&](int j, int buf, bool first) {
-        const uint32_t v_addr = smem_u32(sv + (j % VS) * kTileBytes);
-        const uint32_t a = tmem + kColS + (uint32_t)buf * BN;  // P lies over S
-        const uint32_t o = tmem + kColO + (uint32_t)buf * HD;
-#pragma unroll
-        for (int kk = 0; kk < BN / 16; ++kk)
-          umma_ts(o, a + 8u * kk,
-                  smem_desc_sw128(v_addr + (uint32_t)kk * 2048u, kHalfBytes, 1024), idesc_o,
-                  (!first || kk > 0) ? 1u : 0u);
-        umma_commit(pv_done + buf);
       };
       auto wait_k = [&](int j) {
         if (ok && !mbar_wait(k_full + j % KS, (uint32_t)(j / KS) & 1u, abort_flag, p.spin_limit)) ok = false;
@@ -276,8 +373,13 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
           if (!mbar_wait(p_ready + (j & 1), (uint32_t)(j >> 1) & 1u, abort_flag, p.spin_limit)) { ok = false; break; }
           if (!mbar_wait(v_full + j % VS, (uint32_t)(j / VS) & 1u, abort_flag, p.spin_limit)) { ok = false; break; }
           tc_fence_after_sync();
-          issue_pv(j, j & 1, j < 2);
+          // O_w (+)= P[:, 64 w .. 64 w + 63] V[64 w .. 64 w + 63, :] for both warpgroups' halves
+          const uint32_t a = tmem + kColS + (uint32_t)(j & 1) * BN;
+          const uint32_t vj = v_lo + (uint32_t)(j % VS) * (kTileBytes >> 4);
+          umma_ts_k64(tmem + kColO, a, vj, hi, idesc_o, j > 0 ? 1u : 0u);
+          umma_ts_k64(tmem + kColO + HD, a + 64u, vj + 4u * 128u, hi, idesc_o, j > 0 ? 1u : 0u);
           umma_commit(v_empty + j % VS);
+          umma_commit(pv_done);
           if (j + 2 < T) s_tile(j + 2);
         }
       } else {
@@ -294,7 +396,9 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
           for (int q = 0; q < 2 && ok; ++q) {
             if (!mbar_wait(p_ready + q, (uint32_t)j & 1u, abort_flag, p.spin_limit)) { ok = false; break; }
             tc_fence_after_sync();
-            issue_pv(j, q, j == 0);
+            umma_ts_k128(tmem + kColO + (uint32_t)q * HD, tmem + kColS + (uint32_t)q * BN,
+                         v_lo + (uint32_t)(j % VS) * (kTileBytes >> 4), hi, idesc_o, j > 0 ? 1u : 0u);
+            umma_commit(pv_done + q);
             if (j + 1 < T) issue_s(j + 1, q, q);  // after PV: P of this tile has been consumed
           }
           if (!ok) break;
@@ -306,8 +410,6 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
   } else if (T > 0) {
     // ------------------------------------------------------------- softmax --
     const int quad = warp & 3;               // TMEM lane quadrant this warp may touch
-    // NQ = 1: warpgroup 0 takes the even key tiles, 1 the odd ones, same rows;
-    // NQ = 2: warpgroup q takes every key tile for the rows of M-tile q
     const int wg = (warp - 2) >> 2;
     const int r = quad * 32 + lane;          // row of the M-tile
     const int nl_tile = nl0 + (NQ == 2 ? wg * p.TNL : 0);  // first (node, position) of the rows
@@ -317,128 +419,134 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int hh = r % p.group;
     const int node = min(nl, p.NL - 1) / p.L;
     const uint32_t lane_base = (uint32_t)(quad * 32);
-    // With only a few key tiles the hand-over between the warpgroups costs more
-    // than it hides: warpgroup 0 then works alone ("solo") on both buffers, with
-    // one (maximum, sum, tile count) per buffer, and warpgroup 1 sits the CTA out.
-    const bool solo = NQ == 1 && T <= kSoloTiles;
     const float k2 = p.scale_log2;
-    float m_run = -INFINITY, l_run = 0.f;  // state of the buffer in hand
-    float m_alt = -INFINITY, l_alt = 0.f;  // solo: state of the other buffer
+    float m_run = -INFINITY, l_run = 0.f;  // reference maximum (log2 units) and sum of this thread's accumulator
     bool ok = true;
-    int mine = 0, mine_alt = 0;  // tiles finished on the buffer in hand / on the other one
-    const int j_step = (NQ == 1 && !solo) ? 2 : 1;
-    for (int j = (NQ == 1 && !solo) ? wg : 0; j < T && !(solo && wg == 1); j += j_step) {
-      const int bi = solo ? (j & 1) : wg;                // S/P buffer and accumulator of this tile
-      const uint32_t col_s = kColS + (uint32_t)bi * BN;
-      const uint32_t col_o = kColO + (uint32_t)bi * HD;
-      // wait outcomes are made warp-uniform: the TMEM accesses below are warp-collective
-      if (!__all_sync(0xffffffffu, mbar_wait(s_full + bi, (uint32_t)mine & 1u, abort_flag, p.spin_limit))) {
-        ok = false;
-        break;
-      }
+    // this thread's accumulator: NQ = 1 columns half wg of every tile, NQ = 2 all of M-tile wg
+    const uint32_t col_o = kColO + (uint32_t)wg * HD;
+    uint64_t* my_pv_done = NQ == 1 ? pv_done : pv_done + wg;
+
+    // O *= corr once the products that still write to it have completed
+    auto rescale_o = [&](int j, float corr) -> bool {
+      if (!__all_sync(0xffffffffu, mbar_wait(my_pv_done, (uint32_t)(j - 1) & 1u, abort_flag, p.spin_limit)))
+        return false;
       tc_fence_after_sync();
-      uint32_t s[BN];
-      tmem_ld_x128(tmem_addr(tmem, lane_base, col_s), s);
-      // visible columns of this row in this tile: [lo, hi)
-      const int t = t_begin + j;
-      int lo, hi;
-      if (t < p.TP) {
-        lo = 0;
-        hi = min(BN, p.P - t * BN);
-      } else {
-        lo = node * p.L - (kb_start + (t - p.TP) * BN);
-        hi = lo + p.L;
-      }
-      if (!(lo <= 0 && hi >= BN)) {
 #pragma unroll
-        for (int c = 0; c < BN; ++c)
-          s[c] = (c >= lo && c < hi) ? s[c] : 0xff800000u;  // -inf
-      }
-      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+      for (int c0 = 0; c0 < HD; c0 += 32) {
+        uint32_t o[32];
+        tmem_ld_x32(tmem_addr(tmem, lane_base, col_o + c0), o);
 #pragma unroll
-      for (int c = 0; c < BN; c += 4) {
-        mx0 = fmaxf(mx0, __uint_as_float(s[c]));
-        mx1 = fmaxf(mx1, __uint_as_float(s[c + 1]));
-        mx2 = fmaxf(mx2, __uint_as_float(s[c + 2]));
-        mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
+        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * corr);
+        tmem_st_x32(tmem_addr(tmem, lane_base, col_o + c0), o);
       }
-      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-      const float m_new = fmaxf(m_run, mx * k2);
-      const bool need = (m_new - m_run) > kRescaleLog2;  // false when both are -inf
-      if (__any_sync(0xffffffffu, need)) {
-        float corr = 1.f;
-        if (need) {
-          corr = ex2(m_run - m_new);  // 0 for a row that had seen nothing yet
-          l_run *= corr;
-          m_run = m_new;
+      tmem_wait_st();
+      return true;
+    };
+
+    if constexpr (NQ == 1) {
+      const int half0 = 64 * wg;  // first tile column of this warpgroup's half
+      if (pair) cluster_wait();  // phase 1: the peer's barriers exist
+      for (int j = 0; j < T; ++j) {
+        const int bi = j & 1;
+        const uint32_t col_s = kColS + (uint32_t)bi * BN + (uint32_t)half0;
+        // wait outcomes are made warp-uniform: the TMEM accesses below are warp-collective
+        if (!__all_sync(0xffffffffu, mbar_wait(s_full + bi, (uint32_t)(j >> 1) & 1u, abort_flag, p.spin_limit))) {
+          ok = false;
+          break;
         }
-        if (mine > 0) {  // the accumulator holds this warpgroup's earlier tiles: wait, then rescale
-          if (!__all_sync(0xffffffffu,
-                          mbar_wait(pv_done + bi, (uint32_t)(mine - 1) & 1u, abort_flag, p.spin_limit))) {
+        tc_fence_after_sync();
+        // the last S has been formed: the Q tile and the first K stage are free for the peer's partial
+        if (pair && j == T - 1 && warp == 2 && lane == 0)
+          mbar_arrive_remote(map_to_cta(smem_u32(xchg_ready), (uint32_t)split ^ 1u));
+        uint32_t s[64];
+        tmem_ld_x64(tmem_addr(tmem, lane_base, col_s), s);
+        Window w = visible_window(p, t_begin + j, kb_start, node);
+        const int lo = w.lo - half0, hi = w.hi - half0;  // relative to the half: columns [0, 64)
+        // 32-column chunks that no row of the warp sees cost nothing but zeros in P
+        const bool need0 = __any_sync(0xffffffffu, lo < 32 && hi > 0);
+        const bool need1 = __any_sync(0xffffffffu, lo < 64 && hi > 32);
+        if (!(lo <= 0 && hi >= 64)) {
+#pragma unroll
+          for (int c = 0; c < 64; ++c)
+            s[c] = (c >= lo && c < hi) ? s[c] : 0xff800000u;  // -inf
+        }
+        const uint32_t chunks = (need0 ? 1u : 0u) | (need1 ? 2u : 0u);
+        const float mx = row_max<64>(s, chunks);
+        const float m_new = fmaxf(m_run, mx * k2);
+        const bool need = (m_new - m_run) > kRescaleLog2;  // false when both are -inf
+        if (__any_sync(0xffffffffu, need)) {
+          float corr = 1.f;
+          if (need) {
+            corr = ex2(m_run - m_new);  // 0 for a row that had seen nothing yet
+            l_run *= corr;
+            m_run = m_new;
+          }
+          if (j > 0 && !rescale_o(j, corr)) {  // the accumulator holds the earlier tiles
             ok = false;
             break;
           }
-          tc_fence_after_sync();
-#pragma unroll
-          for (int c0 = 0; c0 < HD; c0 += 32) {
-            uint32_t o[32];
-            tmem_ld_x32(tmem_addr(tmem, lane_base, col_o + c0), o);
-#pragma unroll
-            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * corr);
-            tmem_st_x32(tmem_addr(tmem, lane_base, col_o + c0), o);
-          }
-          tmem_wait_st();
         }
+        const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+        uint32_t pk[32];
+        l_run += row_exps<64>(s, chunks, k2, m_use, pk);
+        // P goes over the first half of the score columns just read (every thread owns its lane)
+        tmem_st_x32(tmem_addr(tmem, lane_base, col_s), pk);
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(p_ready + bi);
       }
-      const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-      uint32_t pk[BN / 2];
-      float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+    } else {
+      for (int j = 0; j < T; ++j) {
+        const uint32_t col_s = kColS + (uint32_t)wg * BN;
+        if (!__all_sync(0xffffffffu, mbar_wait(s_full + wg, (uint32_t)j & 1u, abort_flag, p.spin_limit))) {
+          ok = false;
+          break;
+        }
+        tc_fence_after_sync();
+        uint32_t s[BN];
+        tmem_ld_x128(tmem_addr(tmem, lane_base, col_s), s);
+        const Window w = visible_window(p, t_begin + j, kb_start, node);
+        if (!(w.lo <= 0 && w.hi >= BN)) {
 #pragma unroll
-      for (int c = 0; c < BN; c += 4) {
-        const float p0 = ex2(fmaf(__uint_as_float(s[c]), k2, -m_use));
-        const float p1 = ex2(fmaf(__uint_as_float(s[c + 1]), k2, -m_use));
-        const float p2 = ex2(fmaf(__uint_as_float(s[c + 2]), k2, -m_use));
-        const float p3 = ex2(fmaf(__uint_as_float(s[c + 3]), k2, -m_use));
-        sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
-        pk[c >> 1] = pack_bf16(p0, p1);
-        pk[(c >> 1) + 1] = pack_bf16(p2, p3);
-      }
-      l_run += (sum0 + sum1) + (sum2 + sum3);
-      // P goes over the first half of the S columns just read (every thread owns its lane)
-      tmem_st_x64(tmem_addr(tmem, lane_base, col_s), pk);
-      tmem_wait_st();
-      tc_fence_before_sync();
-      mbar_arrive(p_ready + bi);
-      ++mine;
-      if (solo) {  // the other buffer is next
-        float t = m_run; m_run = m_alt; m_alt = t;
-        t = l_run; l_run = l_alt; l_alt = t;
-        const int c = mine; mine = mine_alt; mine_alt = c;
+          for (int c = 0; c < BN; ++c)
+            s[c] = (c >= w.lo && c < w.hi) ? s[c] : 0xff800000u;  // -inf
+        }
+        const float mx = row_max<BN>(s, 0xfu);
+        const float m_new = fmaxf(m_run, mx * k2);
+        const bool need = (m_new - m_run) > kRescaleLog2;  // false when both are -inf
+        if (__any_sync(0xffffffffu, need)) {
+          float corr = 1.f;
+          if (need) {
+            corr = ex2(m_run - m_new);  // 0 for a row that had seen nothing yet
+            l_run *= corr;
+            m_run = m_new;
+          }
+          if (j > 0 && !rescale_o(j, corr)) {
+            ok = false;
+            break;
+          }
+        }
+        const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+        uint32_t pk[BN / 2];
+        l_run += row_exps<BN>(s, 0xfu, k2, m_use, pk);
+        tmem_st_x64(tmem_addr(tmem, lane_base, col_s), pk);
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(p_ready + wg);
       }
     }
-    // solo: "in hand" is now buffer T & 1; name the two by buffer instead
-    const int buf_hand = solo ? (T & 1) : wg;
-    const uint32_t col_s = kColS + (uint32_t)buf_hand * BN;
-    const uint32_t col_o = kColO + (uint32_t)buf_hand * HD;
     // ------------------------------------------------------------ epilogue --
-    // Each warpgroup waits for its own accumulator, the two exchange their
-    // (reference maximum, sum) per row through two spare tensor-memory columns
-    // of their S buffers, and each then merges and stores one half of the
-    // columns of every row.
-    if (ok && mine > 0)
-      ok = __all_sync(0xffffffffu,
-                      mbar_wait(pv_done + buf_hand, (uint32_t)(mine - 1) & 1u, abort_flag, p.spin_limit));
-    if (ok && solo && mine_alt > 0)
-      ok = __all_sync(0xffffffffu, mbar_wait(pv_done + (buf_hand ^ 1), (uint32_t)(mine_alt - 1) & 1u,
-                                             abort_flag, p.spin_limit));
+    // every product into this thread's accumulator has completed
+    if (ok)
+      ok = __all_sync(0xffffffffu, mbar_wait(my_pv_done, (uint32_t)(T - 1) & 1u, abort_flag, p.spin_limit));
+    __nv_bfloat16* dst =
+        p.out + (((int64_t)b * p.NL + nl) * p.Hq + (int64_t)g * p.group + hh) * HD;
     if constexpr (NQ == 2) {
       // each warpgroup owns its rows outright: normalise (or hand on the partial) and store
       if (ok) {
         tc_fence_after_sync();
         const float inv = p.splits == 1 ? 1.0f / l_run : 1.0f;
         const int64_t tile = ((int64_t)split * gridDim.y + bg) * p.MT + mt + wg;
-        __nv_bfloat16* dst =
-            p.out + (((int64_t)b * p.NL + nl) * p.Hq + (int64_t)g * p.group + hh) * HD;
         float* po = p.part_o + (tile * BM + r) * HD;
 #pragma unroll
         for (int c0 = 0; c0 < HD; c0 += 32) {
@@ -469,128 +577,129 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         }
       }
     } else {
-    const bool active = !(solo && wg == 1);
-    const bool pair = p.pair != 0;
-    float m_o = m_alt, l_o = l_alt;  // state of the other buffer
-    if (!solo) {
-      constexpr uint32_t kColMl = BN / 2;  // first S column that no P lies over
-      tmem_st_x2(tmem_addr(tmem, lane_base, col_s + kColMl), __float_as_uint(m_run),
+      // The two warpgroups exchange their (reference maximum, sum) per row through
+      // spare columns of the first S buffer (every product has completed), and
+      // each then merges and stores one half of the output columns of every row.
+      constexpr uint32_t kColMl = kColS + 32;  // S columns 32..63 hold no P
+      tmem_st_x2(tmem_addr(tmem, lane_base, kColMl + 2u * (uint32_t)wg), __float_as_uint(m_run),
                  __float_as_uint(l_run));
       tmem_wait_st();
       tc_fence_before_sync();
       asm volatile("bar.sync 1, 256;" ::: "memory");  // all eight softmax warps, whatever `ok` says
       tc_fence_after_sync();
       uint32_t um, ul;
-      tmem_ld_x2(tmem_addr(tmem, lane_base, kColS + (uint32_t)(wg ^ 1) * BN + kColMl), um, ul);
-      m_o = __uint_as_float(um);
-      l_o = __uint_as_float(ul);
-    }
-    const float m_a = buf_hand == 0 ? m_run : m_o, l_a = buf_hand == 0 ? l_run : l_o;
-    const float m_b = buf_hand == 0 ? m_o : m_run, l_b = buf_hand == 0 ? l_o : l_run;
-    const float m_all = fmaxf(m_a, m_b);
-    // an accumulator whose warpgroup saw no key of this row (or no tile at all) is left out
-    const bool has_a = m_a != -INFINITY, has_b = m_b != -INFINITY;
-    const float w_a = has_a ? ex2(m_a - m_all) : 0.f;
-    const float w_b = has_b ? ex2(m_b - m_all) : 0.f;
-    const float l_all = w_a * l_a + w_b * l_b;
-    // 32 columns of this CTA's two accumulators, merged against m_all and scaled by f
-    auto merged = [&](int c0, float f, float (&o)[32]) {
-      uint32_t oa[32], ob[32];
-      tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + c0), oa);
-      tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + HD + c0), ob);
-      const float f_a = w_a * f, f_b = w_b * f;
+      tmem_ld_x2(tmem_addr(tmem, lane_base, kColMl + 2u * (uint32_t)(wg ^ 1)), um, ul);
+      const float m_o = __uint_as_float(um), l_o = __uint_as_float(ul);
+      const float m_a = wg == 0 ? m_run : m_o, l_a = wg == 0 ? l_run : l_o;
+      const float m_b = wg == 0 ? m_o : m_run, l_b = wg == 0 ? l_o : l_run;
+      const float m_all = fmaxf(m_a, m_b);
+      // an accumulator whose half held no visible key of this row is left out
+      const bool has_a = m_a != -INFINITY, has_b = m_b != -INFINITY;
+      const float w_a = has_a ? ex2(m_a - m_all) : 0.f;
+      const float w_b = has_b ? ex2(m_b - m_all) : 0.f;
+      const float l_all = w_a * l_a + w_b * l_b;
+      // 32 columns of this CTA's two accumulators, merged against m_all and scaled by f
+      auto merged = [&](int c0, float f, float (&o)[32]) {
+        uint32_t oa[32], ob[32];
+        tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + c0), oa);
+        tmem_ld_x32(tmem_addr(tmem, lane_base, kColO + HD + c0), ob);
+        const float f_a = w_a * f, f_b = w_b * f;
 #pragma unroll
-      for (int c = 0; c < 32; ++c)
-        o[c] = (has_a ? __uint_as_float(oa[c]) * f_a : 0.f) +
-               (has_b ? __uint_as_float(ob[c]) * f_b : 0.f);
-    };
-    auto store_bf16 = [&](__nv_bfloat16* at, const float (&o)[32]) {
+        for (int c = 0; c < 32; ++c)
+          o[c] = (has_a ? __uint_as_float(oa[c]) * f_a : 0.f) +
+                 (has_b ? __uint_as_float(ob[c]) * f_b : 0.f);
+      };
+      auto store_bf16 = [&](__nv_bfloat16* at, const float (&o)[32]) {
 #pragma unroll
-      for (int c = 0; c < 32; c += 8) {
-        uint4 w;
-        w.x = pack_bf16(o[c], o[c + 1]);
-        w.y = pack_bf16(o[c + 2], o[c + 3]);
-        w.z = pack_bf16(o[c + 4], o[c + 5]);
-        w.w = pack_bf16(o[c + 6], o[c + 7]);
-        *reinterpret_cast<uint4*>(at + c) = w;
-      }
-    };
-    __nv_bfloat16* dst =
-        p.out + (((int64_t)b * p.NL + nl) * p.Hq + (int64_t)g * p.group + hh) * HD;
-    if (pair) {
-      // The other half of the key tiles went to the peer CTA of the cluster.  Each of the
-      // two finishes 64 of the 128 columns: it sends its partial of the peer's columns
-      // into the peer's shared memory (the Q tile, idle by then) and merges what it gets.
-      const uint32_t rank = (uint32_t)split, peer = rank ^ 1u;
-      const int cc0 = solo ? 0 : wg, cc1 = solo ? 2 : wg + 1;  // 32-column chunks of a half
-      cluster_sync_all();  // both CTAs have finished their products: Q and K tiles are idle
-      if (active && ok) {
-        tc_fence_after_sync();
-        const uint32_t q_peer = map_to_cta(smem_u32(sq), peer);
-        for (int cc = cc0; cc < cc1; ++cc) {
-          float o[32];
-          merged(64 * (int)peer + 32 * cc, 1.0f, o);
-#pragma unroll
-          for (int k = 0; k < 8; ++k)  // 16-byte chunk (8 cc + k) of row r: chunk-major, rows contiguous
-            st_cluster_f4(q_peer + (uint32_t)(8 * cc + k) * 2048u + (uint32_t)r * 16u, o[4 * k],
-                          o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
+        for (int c = 0; c < 32; c += 8) {
+          uint4 w;
+          w.x = pack_bf16(o[c], o[c + 1]);
+          w.y = pack_bf16(o[c + 2], o[c + 3]);
+          w.z = pack_bf16(o[c + 4], o[c + 5]);
+          w.w = pack_bf16(o[c + 6], o[c + 7]);
+          *reinterpret_cast<uint4*>(at + c) = w;
         }
-        if (solo || wg == 0) st_cluster_f2(map_to_cta(smem_u32(sk), peer) + (uint32_t)r * 8u, m_all, l_all);
-      }
-      cluster_sync_all();  // the peer's partial has arrived
-      if (active && ok) {
-        const float2 mlp = *reinterpret_cast<const float2*>(sk + r * 8);
-        const float m_p = mlp.x, l_p = mlp.y;
-        const float m_fin = fmaxf(m_all, m_p);
-        const float w_l = m_all != -INFINITY ? ex2(m_all - m_fin) : 0.f;
-        const float w_p = m_p != -INFINITY ? ex2(m_p - m_fin) : 0.f;
-        const float inv = 1.0f / (w_l * l_all + w_p * l_p);
-        for (int cc = cc0; cc < cc1; ++cc) {
+      };
+      if (pair) {
+        // The other half of the key tiles went to the peer CTA of the cluster.  Each of the
+        // two finishes 64 of the 128 output columns: it sends its partial of the peer's
+        // columns into the peer's shared memory (the Q tile and the first K stage, idle
+        // since the last S) and merges what it gets.  Hand-over by mbarriers: xchg_ready =
+        // "my buffers are free" (sent from the tile loop), xchg_full = "your partial has
+        // landed", completed by the byte count of the asynchronous stores themselves.
+        const uint32_t rank = (uint32_t)split, peer = rank ^ 1u;
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait_cluster(xchg_ready, 0, abort_flag, p.spin_limit));
+        if (ok) {
+          tc_fence_after_sync();
+          const uint32_t q_peer = map_to_cta(smem_u32(sq), peer);
+          const uint32_t bar_peer = map_to_cta(smem_u32(xchg_full), peer);
           float o[32];
-          merged(64 * (int)rank + 32 * cc, w_l * inv, o);
+          merged(64 * (int)peer + 32 * wg, 1.0f, o);
+#pragma unroll
+          for (int k = 0; k < 8; ++k)  // 16-byte chunk (8 wg + k) of row r: chunk-major, rows contiguous
+            st_async_f4(q_peer + (uint32_t)(8 * wg + k) * 2048u + (uint32_t)r * 16u, bar_peer, o[4 * k],
+                        o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
+          if (wg == 0) st_async_f2(map_to_cta(smem_u32(sk), peer) + (uint32_t)r * 8u, bar_peer, m_all, l_all);
+        }
+        cluster_arrive();  // phase 2: this thread issues nothing more towards the peer
+        // this CTA's own share of its output columns, read while the peer's partial travels
+        float o[32];
+        merged(64 * (int)rank + 32 * wg, 1.0f, o);
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait_cluster(xchg_full, 0, abort_flag, p.spin_limit));
+        if (ok) {
+          const float2 mlp = *reinterpret_cast<const float2*>(sk + r * 8);
+          const float m_p = mlp.x, l_p = mlp.y;
+          const float m_fin = fmaxf(m_all, m_p);
+          const float w_l = m_all != -INFINITY ? ex2(m_all - m_fin) : 0.f;
+          const float w_p = m_p != -INFINITY ? ex2(m_p - m_fin) : 0.f;
+          const float inv = 1.0f / (w_l * l_all + w_p * l_p);
+          const float f_l = w_l * inv, f_p = w_p * inv;
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
-            const float4 q4 = *reinterpret_cast<const float4*>(sq + (8 * cc + k) * 2048 + r * 16);
-            if (w_p != 0.f) {
-              o[4 * k] += q4.x * (w_p * inv);
-              o[4 * k + 1] += q4.y * (w_p * inv);
-              o[4 * k + 2] += q4.z * (w_p * inv);
-              o[4 * k + 3] += q4.w * (w_p * inv);
+            const float4 q4 = *reinterpret_cast<const float4*>(sq + (8 * wg + k) * 2048 + r * 16);
+            o[4 * k] = o[4 * k] * f_l + (w_p != 0.f ? q4.x * f_p : 0.f);
+            o[4 * k + 1] = o[4 * k + 1] * f_l + (w_p != 0.f ? q4.y * f_p : 0.f);
+            o[4 * k + 2] = o[4 * k + 2] * f_l + (w_p != 0.f ? q4.z * f_p : 0.f);
+            o[4 * k + 3] = o[4 * k + 3] * f_l + (w_p != 0.f ? q4.w * f_p : 0.f);
+          }
+          if (row_ok) store_bf16(dst + 64 * (int)rank + 32 * wg, o);
+        }
+      } else if (ok) {
+        tc_fence_after_sync();
+        const float inv = p.splits == 1 ? 1.0f / l_all : 1.0f;
+        const int64_t tile = ((int64_t)split * gridDim.y + bg) * p.MT + mt;
+        float* po = p.part_o + (tile * BM + r) * HD;
+        for (int c0 = wg * 64; c0 < wg * 64 + 64; c0 += 32) {  // each warpgroup stores one half
+          float o[32];
+          merged(c0, inv, o);
+          if (row_ok) {
+            if (p.splits == 1) {
+              store_bf16(dst + c0, o);
+            } else {
+#pragma unroll
+              for (int c = 0; c < 32; c += 4)
+                *reinterpret_cast<float4*>(po + c0 + c) = make_float4(o[c], o[c + 1], o[c + 2], o[c + 3]);
             }
           }
-          if (row_ok) store_bf16(dst + 64 * (int)rank + 32 * cc, o);
+        }
+        if (p.splits > 1 && row_ok && wg == 0) {
+          float* pml = p.part_ml + (tile * BM + r) * 2;
+          pml[0] = m_all;
+          pml[1] = l_all;
         }
       }
-    } else if (active && ok) {
-      const float inv = p.splits == 1 ? 1.0f / l_all : 1.0f;
-      const int64_t tile = ((int64_t)split * gridDim.y + bg) * p.MT + mt;
-      float* po = p.part_o + (tile * BM + r) * HD;
-      // solo: all 128 columns; otherwise each warpgroup stores one half
-      for (int c0 = solo ? 0 : wg * 64; c0 < (solo ? HD : wg * 64 + 64); c0 += 32) {
-        float o[32];
-        merged(c0, inv, o);
-        if (row_ok) {
-          if (p.splits == 1) {
-            store_bf16(dst + c0, o);
-          } else {
-#pragma unroll
-            for (int c = 0; c < 32; c += 4)
-              *reinterpret_cast<float4*>(po + c0 + c) = make_float4(o[c], o[c + 1], o[c + 2], o[c + 3]);
-          }
-        }
-      }
-      if (p.splits > 1 && row_ok && wg == 0) {
-        float* pml = p.part_ml + (tile * BM + r) * 2;
-        pml[0] = m_all;
-        pml[1] = l_all;
-      }
-    }
     }  // NQ == 1
   }
 
-  if (NQ == 1 && p.pair && (warp < 2 || T <= 0)) {
-    cluster_sync_all();  // the two barriers of the paired epilogue
-    cluster_sync_all();
+  if (pair) {
+    // No CTA of the pair leaves while the other may still write into its shared
+    // memory or arrive on its barriers: a second phase of the cluster barrier
+    // (the softmax warps have arrived on it in the epilogue).
+    if (warp < 2 || T <= 0) {
+      cluster_wait();  // phase 1
+      cluster_arrive();
+    }
+    cluster_wait();
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -720,6 +829,7 @@ spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q, cons
   p.part_ml = p.part_o ? p.part_o + (size_t)pl.splits * pl.tiles * BM * HD : nullptr;
   p.status = dev_status;
   p.spin_limit = mbar_poll_limit();
+  p.early_trigger = (d.kernel & SPIFFY_ATTN_EARLY_DEPENDENTS) ? 1 : 0;
 
   if (cudaFuncSetAttribute(graph_attention_tc_kernel<1>,
                            cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||

@@ -29,26 +29,6 @@ struct __align__(16) Partial {
   int pad;
 };
 
-// Two fp32 lanes in one 64-bit register: Blackwell issues their multiply-add and
-// their add as one instruction each (the kernel is bound by instruction issue).
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t r;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-  return r;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
 // acc += {2^(x0 * log2e - ml), 2^(x1 * log2e - ml)}; k2 = {log2e, log2e}, nml2 = {-ml, -ml}
 __device__ __forceinline__ uint64_t add_exp2(uint64_t acc, float x0, float x1, uint64_t k2,
                                              uint64_t nml2) {

@@ -90,6 +90,58 @@ __device__ __forceinline__ void cluster_sync_all() {
                "barrier.cluster.wait.acquire;\n" ::
                    : "memory");
 }
+// The two halves of the cluster barrier: a thread that has arrived may go on
+// with work that does not depend on the other CTAs and wait later.  Every
+// thread of every CTA of the cluster takes part in each phase.
+__device__ __forceinline__ void cluster_arrive() {
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+// One arrival on an mbarrier of another CTA of the cluster (`addr` from
+// map_to_cta); orders this thread's earlier writes, also those into that CTA's
+// shared memory, before the arrival.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(addr) : "memory");
+}
+// 16 bytes into another CTA's shared memory without waiting for them: the
+// destination CTA's mbarrier `bar` (same CTA as `addr`) counts the bytes as a
+// transaction, so whoever waits on it with the byte count expected sees them.
+__device__ __forceinline__ void st_async_f4(uint32_t addr, uint32_t bar, float a, float b, float c, float d) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%2, %3, %4, %5}, [%1];"
+               ::"r"(addr), "r"(bar), "f"(a), "f"(b), "f"(c), "f"(d)
+               : "memory");
+}
+__device__ __forceinline__ void st_async_f2(uint32_t addr, uint32_t bar, float a, float b) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%2, %3}, [%1];"
+               ::"r"(addr), "r"(bar), "f"(a), "f"(b)
+               : "memory");
+}
+// try_wait that also acquires what threads of other CTAs released with
+// mbar_arrive_remote.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort,
+                                                  uint32_t limit) {
+  for (uint32_t i = 0; i < limit; ++i) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if ((i & 15u) == 15u && *abort) return false;
+  }
+  *abort = 1;
+  return false;
+}
 // The address, in the shared window of the cluster, of `smem_addr` in CTA `rank`.
 __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
   uint32_t r;
@@ -140,6 +192,17 @@ __device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t (&r)[32]) {
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
       "tcgen05.wait::ld.sync.aligned;\n"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+
+// Row `lane` of the warp's TMEM quadrant, 64 consecutive 32-bit columns from
+// `taddr`, into r[0..63]; returns once the data has arrived.
+__device__ __forceinline__ void tmem_ld_x64(uint32_t taddr, uint32_t (&r)[64]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%64];\n"
+      "tcgen05.wait::ld.sync.aligned;\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
       : "r"(taddr)
       : "memory");
 }
@@ -245,6 +308,154 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
       : "r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// ------------------------------------------------- lean issue of MMA groups --
+// One thread issues every MMA of a CTA; what it spends per instruction on
+// building descriptors bounds the tensor pipe's rate (a 128 x 128 x 16 product
+// lasts 64 cycles).  The groups below take the descriptors split into their low
+// word (address and leading offset: advanced by a constant per K step) and
+// their high word (stride offset, fixed bits, swizzle: the same for all).
+__device__ __forceinline__ uint32_t desc_lo_sw128(uint32_t addr, uint32_t lbo_bytes) {
+  return ((addr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
+}
+__host__ __device__ constexpr uint32_t desc_hi_sw128(uint32_t sbo_bytes) {
+  return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);
+}
+// D[tmem] (+)= A B^T over K = 128: A and B K-major tiles of 128-byte-swizzled
+// rows, stored as two 64-element halves 16 KB apart (eight K steps of 16).
+__device__ __forceinline__ void umma_ss_k128(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi,
+                                             uint32_t idesc, uint32_t accumulate_first) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p0, p1;\n"
+      ".reg .b32 al, bl;\n"
+      ".reg .b64 da, db;\n"
+      "setp.ne.b32 p0, %5, 0;\n"
+      "setp.eq.b32 p1, %5, %5;\n"
+      "add.u32 al, %1, 0;\n"
+      "add.u32 bl, %2, 0;\n"
+      "mov.b64 da, {al, %3};\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p0;\n"
+      "add.u32 al, %1, 2;\n"
+      "add.u32 bl, %2, 2;\n"
+      "mov.b64 da, {al, %3};\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n"
+      "add.u32 al, %1, 4;\n"
+      "add.u32 bl, %2, 4;\n"
+      "mov.b64 da, {al, %3};\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n"
+      "add.u32 al, %1, 6;\n"
+      "add.u32 bl, %2, 6;\n"
+      "mov.b64 da, {al, %3};\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n"
+      "add.u32 al, %1, 1024;\n"
+      "add.u32 bl, %2, 1024;\n"
+      "mov.b64 da, {al, %3};\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n"
+      "add.u32 al, %1, 1026;\n"
+      "add.u32 bl, %2, 1026;\n"
+      "mov.b64 da, {al, %3};\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n"
+      "add.u32 al, %1, 1028;\n"
+      "add.u32 bl, %2, 1028;\n"
+      "mov.b64 da, {al, %3};\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n"
+      "add.u32 al, %1, 1030;\n"
+      "add.u32 bl, %2, 1030;\n"
+      "mov.b64 da, {al, %3};\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n"
+      "}\n"
+      :
+      : "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate_first)
+      : "memory");
+}
+// D[tmem] (+)= A[tmem] B over `steps` K steps of 16: A = bf16 pairs in tensor
+// memory (8 columns per step), B an MN-major tile whose rows of 16 keys are
+// 2048 bytes apart.
+__device__ __forceinline__ void umma_ts_k64(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi,
+                                            uint32_t idesc, uint32_t accumulate_first) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p0, p1;\n"
+      ".reg .b32 at, bl;\n"
+      ".reg .b64 db;\n"
+      "setp.ne.b32 p0, %5, 0;\n"
+      "setp.eq.b32 p1, %5, %5;\n"
+      "add.u32 at, %1, 0;\n"
+      "add.u32 bl, %2, 0;\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, p0;\n"
+      "add.u32 at, %1, 8;\n"
+      "add.u32 bl, %2, 128;\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, p1;\n"
+      "add.u32 at, %1, 16;\n"
+      "add.u32 bl, %2, 256;\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, p1;\n"
+      "add.u32 at, %1, 24;\n"
+      "add.u32 bl, %2, 384;\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, p1;\n"
+      "}\n"
+      :
+      : "r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate_first)
+      : "memory");
+}
+__device__ __forceinline__ void umma_ts_k128(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi,
+                                             uint32_t idesc, uint32_t accumulate_first) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p0, p1;\n"
+      ".reg .b32 at, bl;\n"
+      ".reg .b64 db;\n"
+      "setp.ne.b32 p0, %5, 0;\n"
+      "setp.eq.b32 p1, %5, %5;\n"
+      "add.u32 at, %1, 0;\n"
+      "add.u32 bl, %2, 0;\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, p0;\n"
+      "add.u32 at, %1, 8;\n"
+      "add.u32 bl, %2, 128;\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, p1;\n"
+      "add.u32 at, %1, 16;\n"
+      "add.u32 bl, %2, 256;\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, p1;\n"
+      "add.u32 at, %1, 24;\n"
+      "add.u32 bl, %2, 384;\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, p1;\n"
+      "add.u32 at, %1, 32;\n"
+      "add.u32 bl, %2, 512;\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, p1;\n"
+      "add.u32 at, %1, 40;\n"
+      "add.u32 bl, %2, 640;\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, p1;\n"
+      "add.u32 at, %1, 48;\n"
+      "add.u32 bl, %2, 768;\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, p1;\n"
+      "add.u32 at, %1, 56;\n"
+      "add.u32 bl, %2, 896;\n"
+      "mov.b64 db, {bl, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, p1;\n"
+      "}\n"
+      :
+      : "r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate_first)
+      : "memory");
+}
+
 // The mbarrier receives one arrival when every MMA issued so far by this
 // thread has completed (implies tcgen05.fence::before_thread_sync).
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {

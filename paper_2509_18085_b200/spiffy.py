@@ -22,6 +22,7 @@ F32, BF16 = 0, 1
 RULE_TOPS, RULE_THRESHOLD = 0, 1
 DEV_NONFINITE, DEV_BADGRAPH, DEV_TIMEOUT = 1, 2, 4
 ATTN_AUTO, ATTN_SIMT, ATTN_TCGEN05 = 0, 1, 2
+ATTN_EARLY_DEPENDENTS = 0x100  # flag OR-ed into the kernel selection
 
 DECIDE_STATIC_BYTES = 2 << 20
 
