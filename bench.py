@@ -62,7 +62,7 @@ def parse():
     ap.add_argument("--no-other-shapes", action="store_true", help="skip the timing of the other configurations")
     ap.add_argument("--no-early-dependents", action="store_true",
                     help="whole-model step without SPIFFY_ATTN_EARLY_DEPENDENTS on the layers' attention calls")
-    ap.add_argument("--part", default="step", choices=["step", "attention", "decide", "decide_walk", "decide_walk_lazy", "decide_sampled", "lmhead", "draft"],
+    ap.add_argument("--part", default="step", choices=["step", "attention", "full_sequence", "decide", "decide_walk", "decide_walk_lazy", "decide_sampled", "lmhead", "draft"],
                     help="time one library call alone on any configuration (for profiling); "
                          "the benchmark line itself is --part step")
     ap.add_argument("--sets", type=int, default=0, help="rotating input sets for --part (0 = enough to exceed L2)")
@@ -241,6 +241,8 @@ def run_part(args):
         return run_draft_part(args, cfg)
     if args.part == "lmhead":
         return run_lmhead_part(args, cfg)
+    if args.part == "full_sequence":
+        return run_full_sequence_part(args, cfg)
     attn = args.part == "attention"
     probe = W.make(cfg, W.seed_for(args.config, 100), attention=attn, decision=not attn)
     masked = int((probe.block_tokens == cfg.mask_id).sum())
@@ -302,6 +304,42 @@ def run_part(args):
                        note="gbs counts the eager call's bytes (every node); lazy_gbs the bytes this call reads")
     out["peaks"] = peaks["source"]
     print(json.dumps(out))
+
+
+def run_full_sequence_part(args, cfg):
+    """spiffy_full_sequence_attention alone: the configuration's nodes plus three
+    trailing masked blocks as extra queries (Fig. 3 caption, App. A.2)."""
+    import torch
+    from paper_2509_18085_b200 import spiffy
+    B, N, L, P = cfg.batch, cfg.n_nodes, cfg.block_len, cfg.prefix_len
+    S = 3 * L
+    g = torch.Generator(device="cuda").manual_seed(17)
+    r = lambda *shape: torch.randn(shape, generator=g, device="cuda").to(torch.bfloat16)
+    per_set = 2 * B * (2 * (N * L + S) * cfg.n_q_heads + 2 * (P + N * L + S) * cfg.n_kv_heads) * cfg.head_dim
+    n_sets = args.sets or max(2, min(16, int(300e6 // per_set) + 1))
+    sets = [(r(B, N, L, cfg.n_q_heads, cfg.head_dim), r(B, S, cfg.n_q_heads, cfg.head_dim),
+             r(B, P, cfg.n_kv_heads, cfg.head_dim), r(B, P, cfg.n_kv_heads, cfg.head_dim),
+             r(B, S, cfg.n_kv_heads, cfg.head_dim), r(B, S, cfg.n_kv_heads, cfg.head_dim),
+             r(B, N, L, cfg.n_kv_heads, cfg.head_dim), r(B, N, L, cfg.n_kv_heads, cfg.head_dim)) for _ in range(n_sets)]
+    out_n, out_s = spiffy.spiffy_full_sequence_attention(*sets[0])
+    desc = spiffy.attn_desc(sets[0][0], sets[0][2], sets[0][6], 0.0, spiffy.ATTN_TCGEN05)
+    ws = torch.empty(max(16, int(spiffy.lib().spiffy_full_sequence_attention_workspace(
+        __import__("ctypes").byref(desc), S))), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        timer = GraphTimer(stream)
+        fns = [lambda x=x: spiffy.spiffy_full_sequence_attention(*x, out_nodes=out_n, out_suffix=out_s, workspace=ws)
+               for x in sets]
+        for fn in fns:
+            fn()
+        stream.synchronize()
+        sec, replays, _ = timer.measure(timer.capture(fns))
+    sec /= n_sets
+    peaks = measured_peaks()
+    print(json.dumps({"part": "full_sequence", "config": f"config{args.config}-{cfg.name}", "suffix_rows": S,
+                      "us_per_call": sec * 1e6, "launches_per_call": 2, "input_sets": n_sets,
+                      "algorithmic_bytes": per_set, "gbs": per_set / sec / 1e9,
+                      "frac_of_hbm": per_set / sec / 1e9 / peaks["hbm_gbs"], "peaks": peaks["source"]}))
 
 
 def run_lmhead_part(args, cfg):

@@ -11,6 +11,9 @@
  *   spiffy_graph_attention   the packed attention of Sec. 4.3 (mask of Fig. 3):
  *                            every draft state attends to the cached context
  *                            and, bidirectionally, to its own block only;
+ *   spiffy_full_sequence_attention
+ *                            the same with trailing masked blocks as extra
+ *                            queries (full-sequence models, App. A.2);
  *   spiffy_unmask_decide     steps 1-4 of Algorithm 1 (the function Next() of
  *                            App. A) evaluated for every node of the graph;
  *   spiffy_accept_walk       step 5 of Algorithm 1: the walk through the draft
@@ -141,6 +144,34 @@ spiffy_status spiffy_graph_attention(const spiffy_attn_desc* desc,
                                      const void* v_block, void* out,
                                      int32_t* dev_status, void* workspace,
                                      size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The verification attention of a full-sequence bidirectional model that caches
+ * only its prefix (caption of Fig. 3; App. A.2): the block being decoded (node 0)
+ * and the S trailing, still fully masked positions attend to the whole true
+ * sequence -- prefix, true block, suffix --, every draft block to the prefix, the
+ * suffix and itself (every block of the true sequence except the one it is a
+ * draft of).  Two launches of the tensor-core kernel, no copy: the nodes with
+ * the context given as two segments [prefix ; suffix], then the suffix rows as
+ * one node whose block is the suffix and whose context is [prefix ; true block].
+ *
+ *   desc      batch, n_nodes, block_len, prefix_len, heads, head_dim, scale of the
+ *             nodes' call; dtype bf16 and head_dim 128 (else SPIFFY_EUNSUPPORTED)
+ *   suffix_len S in [0, 1024]; 0 makes this spiffy_graph_attention
+ *   q_nodes, out_nodes   [B][N][L][Hq][d]     q_suffix, out_suffix [B][S][Hq][d]
+ *   k/v_prefix [B][P][Hkv][d]   k/v_suffix [B][S][Hkv][d]   k/v_block [B][N][L][Hkv][d]
+ * dev_status, stream and error behaviour as in spiffy_graph_attention; the
+ * workspace (spiffy_full_sequence_attention_workspace) serves both launches.
+ */
+size_t spiffy_full_sequence_attention_workspace(const spiffy_attn_desc* desc, int32_t suffix_len);
+spiffy_status spiffy_full_sequence_attention(const spiffy_attn_desc* desc, int32_t suffix_len,
+                                             const void* q_nodes, const void* q_suffix,
+                                             const void* k_prefix, const void* v_prefix,
+                                             const void* k_suffix, const void* v_suffix,
+                                             const void* k_block, const void* v_block,
+                                             void* out_nodes, void* out_suffix,
+                                             int32_t* dev_status, void* workspace,
+                                             size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------- */
 /* Decision: steps 1-4 of Algorithm 1 for every node (Next() of App. A)      */

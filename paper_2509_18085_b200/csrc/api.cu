@@ -81,7 +81,7 @@ extern "C" {
 
 size_t spiffy_graph_attention_workspace(const spiffy_attn_desc* desc) {
   if (check_attn_desc(desc) != SPIFFY_OK) return 0;
-  return use_tc(*desc) ? attention_tc_workspace_bytes(*desc) : 0;
+  return use_tc(*desc) ? attention_tc_workspace_bytes(*desc, 0) : 0;
 }
 
 spiffy_status spiffy_graph_attention(const spiffy_attn_desc* desc, const void* q,
@@ -100,15 +100,73 @@ spiffy_status spiffy_graph_attention(const spiffy_attn_desc* desc, const void* q
     return SPIFFY_EINVAL;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   if (use_tc(d)) {
-    const size_t need = attention_tc_workspace_bytes(d);
+    const size_t need = attention_tc_workspace_bytes(d, 0);
     if (need > 0 && (!workspace || workspace_bytes < need || !aligned16(workspace)))
       return SPIFFY_EWORKSPACE;
-    return launch_attention_tc(d, q, k_prefix, v_prefix, k_block, v_block, out,
-                               dev_status, workspace, stream);
+    const AttnContext ctx = {k_prefix, v_prefix, d.prefix_len, 0};
+    const AttnContext none = {nullptr, nullptr, 0, 0};
+    return launch_attention_tc(d, q, ctx, none, k_block, v_block, out, dev_status, workspace, stream);
   }
   if ((d.kernel & 0xff) == SPIFFY_ATTN_TCGEN05) return SPIFFY_EUNSUPPORTED;
   if (d.block_len > 64) return SPIFFY_EUNSUPPORTED;  // the CUDA-core kernel keeps a block's rows in registers
   return launch_attention_simt(d, q, k_prefix, v_prefix, k_block, v_block, out, stream);
+}
+
+namespace {
+// The second launch of the full-sequence call: the suffix rows as one node whose block is the suffix.
+spiffy_attn_desc suffix_desc(const spiffy_attn_desc& d, int32_t suffix_len) {
+  spiffy_attn_desc s = d;
+  s.n_nodes = 1;
+  s.block_len = suffix_len;
+  return s;
+}
+spiffy_status check_full_sequence(const spiffy_attn_desc* desc, int32_t suffix_len) {
+  const spiffy_status st = check_attn_desc(desc);
+  if (st != SPIFFY_OK) return st;
+  if (suffix_len < 0) return SPIFFY_EINVAL;
+  if (suffix_len > 1024) return SPIFFY_EUNSUPPORTED;
+  if (!use_tc(*desc)) return SPIFFY_EUNSUPPORTED;  // bf16, head dimension 128 only
+  return SPIFFY_OK;
+}
+}  // namespace
+
+size_t spiffy_full_sequence_attention_workspace(const spiffy_attn_desc* desc, int32_t suffix_len) {
+  if (check_full_sequence(desc, suffix_len) != SPIFFY_OK) return 0;
+  const size_t nodes = attention_tc_workspace_bytes(*desc, suffix_len);
+  const size_t suffix = suffix_len > 0 ? attention_tc_workspace_bytes(suffix_desc(*desc, suffix_len), desc->block_len) : 0;
+  return nodes > suffix ? nodes : suffix;
+}
+
+spiffy_status spiffy_full_sequence_attention(const spiffy_attn_desc* desc, int32_t suffix_len,
+                                             const void* q_nodes, const void* q_suffix,
+                                             const void* k_prefix, const void* v_prefix,
+                                             const void* k_suffix, const void* v_suffix,
+                                             const void* k_block, const void* v_block, void* out_nodes,
+                                             void* out_suffix, int32_t* dev_status, void* workspace,
+                                             size_t workspace_bytes, void* cuda_stream) {
+  const spiffy_status st = check_full_sequence(desc, suffix_len);
+  if (st != SPIFFY_OK) return st;
+  const spiffy_attn_desc d = *desc;
+  if (!q_nodes || !k_block || !v_block || !out_nodes) return SPIFFY_EINVAL;
+  if (d.prefix_len > 0 && (!k_prefix || !v_prefix)) return SPIFFY_EINVAL;
+  if (suffix_len > 0 && (!q_suffix || !k_suffix || !v_suffix || !out_suffix)) return SPIFFY_EINVAL;
+  const void* all[] = {q_nodes, q_suffix, k_prefix, v_prefix, k_suffix, v_suffix, k_block, v_block, out_nodes, out_suffix};
+  for (const void* ptr : all)
+    if (!aligned16(ptr)) return SPIFFY_EINVAL;
+  const size_t need = spiffy_full_sequence_attention_workspace(desc, suffix_len);
+  if (need > 0 && (!workspace || workspace_bytes < need || !aligned16(workspace))) return SPIFFY_EWORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const AttnContext prefix = {k_prefix, v_prefix, d.prefix_len, 0};
+  // nodes: context = [prefix ; suffix]; every node's own block as always
+  const AttnContext suffix = {k_suffix, v_suffix, suffix_len, 0};
+  spiffy_status rc = launch_attention_tc(d, q_nodes, prefix, suffix, k_block, v_block, out_nodes, dev_status,
+                                         workspace, stream);
+  if (rc != SPIFFY_OK || suffix_len == 0) return rc;
+  // suffix rows: one node whose block is the suffix; context = [prefix ; the true block], the
+  // latter being node 0 of every sequence's blocks (sequences N * L rows apart)
+  const AttnContext true_block = {k_block, v_block, d.block_len, (int64_t)d.n_nodes * d.block_len};
+  return launch_attention_tc(suffix_desc(d, suffix_len), q_suffix, prefix, true_block, k_suffix, v_suffix,
+                             out_suffix, dev_status, workspace, stream);
 }
 
 size_t spiffy_unmask_decide_workspace(const spiffy_decide_desc* desc) {

@@ -81,11 +81,12 @@ constexpr int kSmemBytes = Smem<1>::total + 1024;  // slack for 1024-byte alignm
 static_assert(Smem<1>::total == Smem<2>::total, "both layouts use the same amount");
 
 struct Params {
-  int B, N, L, P, Hq, Hkv, group;
+  int B, N, L, Hq, Hkv, group;
+  int P, P2;    // context keys: first and second segment
   int TNL;      // (node, position) pairs per M-tile
   int NL;       // N * L
   int MT;       // M-tiles per (sequence, kv head)
-  int TP;       // context key tiles
+  int TP1, TP;  // context key tiles: of the first segment, of both
   int splits;
   int pair;  // the two splits are the two CTAs of a cluster and merge through shared memory
   float scale_log2;
@@ -172,7 +173,7 @@ __device__ __forceinline__ Window visible_window(const Params& p, int t, int kb_
   Window w;
   if (t < p.TP) {  // context: every row sees every key that exists
     w.lo = 0;
-    w.hi = min(BN, p.P - t * BN);
+    w.hi = t < p.TP1 ? min(BN, p.P - t * BN) : min(BN, p.P2 - (t - p.TP1) * BN);
   } else {  // block keys: the row's own node only
     w.lo = node * p.L - (kb_start + (t - p.TP) * BN);
     w.hi = w.lo + p.L;
@@ -193,6 +194,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                           const __grid_constant__ CUtensorMap tm_kp,
                           const __grid_constant__ CUtensorMap tm_vp,
+                          const __grid_constant__ CUtensorMap tm_kp2,
+                          const __grid_constant__ CUtensorMap tm_vp2,
                           const __grid_constant__ CUtensorMap tm_kb,
                           const __grid_constant__ CUtensorMap tm_vb, const Params p) {
   extern __shared__ uint8_t smem_raw[];
@@ -257,9 +260,11 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     }
     uint64_t* full = (is_k ? k_full : v_full) + stage;
     const int t = t_begin + j;
-    const bool ctx = t < p.TP;
-    const CUtensorMap* m = is_k ? (ctx ? &tm_kp : &tm_kb) : (ctx ? &tm_vp : &tm_vb);
-    const int key0 = ctx ? t * BN : kb_start + (t - p.TP) * BN;
+    // key tiles in order: first context segment, second context segment, block keys
+    const int seg = t < p.TP1 ? 0 : (t < p.TP ? 1 : 2);
+    const CUtensorMap* m = is_k ? (seg == 0 ? &tm_kp : seg == 1 ? &tm_kp2 : &tm_kb)
+                                : (seg == 0 ? &tm_vp : seg == 1 ? &tm_vp2 : &tm_vb);
+    const int key0 = seg == 0 ? t * BN : seg == 1 ? (t - p.TP1) * BN : kb_start + (t - p.TP) * BN;
     uint8_t* dst = (is_k ? sk : sv) + stage * kTileBytes;
     mbar_arrive_expect_tx(full, kTileBytes);
     tma_load_4d(dst, m, full, 0, g, key0, b);
@@ -270,7 +275,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
 
   if (threadIdx.x == 0) {
     prefetch_tensormap(&tm_q);  // the descriptors are kernel parameters
-    prefetch_tensormap(p.TP > 0 ? &tm_kp : &tm_kb);
+    prefetch_tensormap(p.TP1 > 0 ? &tm_kp : (p.TP > 0 ? &tm_kp2 : &tm_kb));
     mbar_init(q_full, 1);
     for (int i = 0; i < KS; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_ready + i, NQ == 1 ? 256 : 128); }
@@ -293,7 +298,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
       while (issued_k < T && produce(true, issued_k, false)) {}
     }
   } else if (threadIdx.x == 32) {
-    prefetch_tensormap(p.TP > 0 ? &tm_vp : &tm_vb);
+    prefetch_tensormap(p.TP1 > 0 ? &tm_vp : (p.TP > 0 ? &tm_vp2 : &tm_vb));
     for (int i = 0; i < VS; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
     mbar_fence_init();
     cudaGridDependencySynchronize();
@@ -750,19 +755,20 @@ graph_attention_combine_kernel(const Params p) {
 
 // ------------------------------------------------------------------ host ----
 struct Plan {
-  int group, TNL, NL, MT, TP, splits;
+  int group, TNL, NL, MT, TP1, TP, splits;
   int nq;    // M-tiles per CTA
   int pair;  // key tiles split over the two CTAs of a cluster (no workspace, no merge kernel)
   int64_t tiles;  // B * Hkv * MT
 };
 
-Plan make_plan(const spiffy_attn_desc& d) {
+Plan make_plan(const spiffy_attn_desc& d, int ctx2_len) {
   Plan pl;
   pl.group = d.n_q_heads / d.n_kv_heads;
   pl.TNL = BM / pl.group;
   pl.NL = d.n_nodes * d.block_len;
   pl.MT = (pl.NL + pl.TNL - 1) / pl.TNL;
-  pl.TP = (d.prefix_len + BN - 1) / BN;
+  pl.TP1 = (d.prefix_len + BN - 1) / BN;
+  pl.TP = pl.TP1 + (ctx2_len + BN - 1) / BN;
   pl.tiles = (int64_t)d.batch * d.n_kv_heads * pl.MT;
   // Two M-tiles per CTA once the paired CTAs still fill the machine: every K/V
   // tile then serves twice as many rows per trip from L2.
@@ -794,33 +800,40 @@ bool attention_tc_supported(const spiffy_attn_desc& d) {
   return true;
 }
 
-size_t attention_tc_workspace_bytes(const spiffy_attn_desc& d) {
-  const Plan pl = make_plan(d);
+size_t attention_tc_workspace_bytes(const spiffy_attn_desc& d, int ctx2_len) {
+  const Plan pl = make_plan(d, ctx2_len);
   if (pl.splits == 1 || pl.pair) return 0;
   return (size_t)pl.splits * pl.tiles * BM * (HD + 2) * sizeof(float);
 }
 
-spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q, const void* kp,
-                                  const void* vp, const void* kb, const void* vb, void* out,
+spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q, const AttnContext& ctx,
+                                  const AttnContext& ctx2, const void* kb, const void* vb, void* out,
                                   int32_t* dev_status, void* ws, cudaStream_t stream) {
-  const Plan pl = make_plan(d);
-  CUtensorMap tm_q, tm_kp, tm_vp, tm_kb, tm_vb;
+  const Plan pl = make_plan(d, ctx2.len);
+  CUtensorMap tm_q, tm_kp, tm_vp, tm_kp2, tm_vp2, tm_kb, tm_vb;
   bool ok = make_map(&tm_q, q, d.n_q_heads, pl.NL, d.batch, pl.group, pl.TNL);
   ok = ok && make_map(&tm_kb, kb, d.n_kv_heads, pl.NL, d.batch, 1, BN);
   ok = ok && make_map(&tm_vb, vb, d.n_kv_heads, pl.NL, d.batch, 1, BN);
-  if (d.prefix_len > 0) {
-    ok = ok && make_map(&tm_kp, kp, d.n_kv_heads, d.prefix_len, d.batch, 1, BN);
-    ok = ok && make_map(&tm_vp, vp, d.n_kv_heads, d.prefix_len, d.batch, 1, BN);
-  } else {  // never dereferenced: there is no context tile
+  if (ctx.len > 0) {
+    ok = ok && make_map(&tm_kp, ctx.k, d.n_kv_heads, ctx.len, d.batch, 1, BN, ctx.batch_stride_rows);
+    ok = ok && make_map(&tm_vp, ctx.v, d.n_kv_heads, ctx.len, d.batch, 1, BN, ctx.batch_stride_rows);
+  } else {  // never dereferenced: the segment has no tile
     tm_kp = tm_kb;
     tm_vp = tm_vb;
+  }
+  if (ctx2.len > 0) {
+    ok = ok && make_map(&tm_kp2, ctx2.k, d.n_kv_heads, ctx2.len, d.batch, 1, BN, ctx2.batch_stride_rows);
+    ok = ok && make_map(&tm_vp2, ctx2.v, d.n_kv_heads, ctx2.len, d.batch, 1, BN, ctx2.batch_stride_rows);
+  } else {
+    tm_kp2 = tm_kb;
+    tm_vp2 = tm_vb;
   }
   if (!ok) return SPIFFY_ECUDA;
 
   Params p;
-  p.B = d.batch; p.N = d.n_nodes; p.L = d.block_len; p.P = d.prefix_len;
+  p.B = d.batch; p.N = d.n_nodes; p.L = d.block_len; p.P = ctx.len; p.P2 = ctx2.len;
   p.Hq = d.n_q_heads; p.Hkv = d.n_kv_heads; p.group = pl.group;
-  p.TNL = pl.TNL; p.NL = pl.NL; p.MT = pl.MT; p.TP = pl.TP; p.splits = pl.splits;
+  p.TNL = pl.TNL; p.NL = pl.NL; p.MT = pl.MT; p.TP1 = pl.TP1; p.TP = pl.TP; p.splits = pl.splits;
   p.pair = pl.pair;
   const float scale = d.scale != 0.f ? d.scale : 1.0f / sqrtf((float)d.head_dim);
   p.scale_log2 = scale * kLog2e;
@@ -853,7 +866,7 @@ spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q, cons
     attr[1].val.clusterDim.z = 2;
     cfg.attrs = attr;
     cfg.numAttrs = pl.pair ? 2 : 1;
-    if (cudaLaunchKernelEx(&cfg, kern, tm_q, tm_kp, tm_vp, tm_kb, tm_vb, p) != cudaSuccess)
+    if (cudaLaunchKernelEx(&cfg, kern, tm_q, tm_kp, tm_vp, tm_kp2, tm_vp2, tm_kb, tm_vb, p) != cudaSuccess)
       return SPIFFY_ECUDA;
   }
   count_launch();

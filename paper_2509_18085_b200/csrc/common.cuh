@@ -128,14 +128,20 @@ spiffy_status launch_draft(const spiffy_draft_desc& d, const void* logits, const
                            int32_t* parent_off, int32_t* parent_idx, int32_t* dev_status, void* ws,
                            cudaStream_t stream);
 
-// tcgen05 path: shape support query, workspace and launch.
+// tcgen05 path: shape support query, workspace and launch.  The cached context
+// comes as up to two segments of keys/values, [B][len][Hkv][d] each, whose
+// sequences may lie `batch_stride_rows` rows apart (0: densely packed).
+struct AttnContext {
+  const void* k;
+  const void* v;
+  int len;
+  int64_t batch_stride_rows;
+};
 bool attention_tc_supported(const spiffy_attn_desc& d);
-size_t attention_tc_workspace_bytes(const spiffy_attn_desc& d);
-spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q,
-                                  const void* kp, const void* vp,
-                                  const void* kb, const void* vb, void* out,
-                                  int32_t* dev_status, void* ws,
-                                  cudaStream_t stream);
+size_t attention_tc_workspace_bytes(const spiffy_attn_desc& d, int ctx2_len);
+spiffy_status launch_attention_tc(const spiffy_attn_desc& d, const void* q, const AttnContext& ctx,
+                                  const AttnContext& ctx2, const void* kb, const void* vb, void* out,
+                                  int32_t* dev_status, void* ws, cudaStream_t stream);
 
 // Launch with programmatic stream serialisation: the kernel may be scheduled
 // while its predecessor in the stream is still draining.  Every kernel launched

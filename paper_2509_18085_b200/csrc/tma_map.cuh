@@ -30,13 +30,16 @@ EncodeTiledFn encode_fn() {
 // Tensor [outer][rows][heads][128] of bf16 (equally: a [rows][heads * 128] matrix) seen as a
 // 4-D TMA tensor with the 64-element half of a head row innermost; box = 64 x box_heads x
 // box_rows x 1.
+// `outer_stride_rows`: rows between consecutive outer slices (0 = densely packed, i.e. `rows`);
+// larger when the tensor is a window of `rows` rows into a longer one.
 bool make_map(CUtensorMap* m, const void* base, int heads, int64_t rows, int outer, int box_heads,
-              int box_rows) {
+              int box_rows, int64_t outer_stride_rows = 0) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return false;
+  if (outer_stride_rows <= 0) outer_stride_rows = rows;
   const cuuint64_t dims[4] = {(cuuint64_t)kMapInner, (cuuint64_t)heads, (cuuint64_t)rows, (cuuint64_t)outer};
   const cuuint64_t strides[3] = {(cuuint64_t)kMapInner * 2, (cuuint64_t)heads * kMapInner * 2,
-                                 (cuuint64_t)rows * heads * kMapInner * 2};
+                                 (cuuint64_t)outer_stride_rows * heads * kMapInner * 2};
   const cuuint32_t box[4] = {64, (cuuint32_t)box_heads, (cuuint32_t)box_rows, 1};
   const cuuint32_t es[4] = {1, 1, 1, 1};
   return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,

@@ -78,6 +78,10 @@ def lib() -> ctypes.CDLL:
         L.spiffy_graph_attention_workspace.argtypes = [ctypes.POINTER(AttnDesc)]
         L.spiffy_graph_attention.restype = ctypes.c_int
         L.spiffy_graph_attention.argtypes = [ctypes.POINTER(AttnDesc)] + [vp] * 8 + [sz, vp]
+        L.spiffy_full_sequence_attention_workspace.restype = sz
+        L.spiffy_full_sequence_attention_workspace.argtypes = [ctypes.POINTER(AttnDesc), i32]
+        L.spiffy_full_sequence_attention.restype = ctypes.c_int
+        L.spiffy_full_sequence_attention.argtypes = [ctypes.POINTER(AttnDesc), i32] + [vp] * 12 + [sz, vp]
         L.spiffy_unmask_decide_workspace.restype = sz
         L.spiffy_unmask_decide_workspace.argtypes = [ctypes.POINTER(DecideDesc)]
         L.spiffy_unmask_decide.restype = ctypes.c_int
@@ -204,31 +208,34 @@ def spiffy_unmask_decide_workspace(desc: DecideDesc) -> int:
 
 
 def spiffy_full_sequence_attention(q_nodes, q_suffix, k_prefix, v_prefix, k_suffix, v_suffix, k_block,
-                                   v_block, scale: float = 0.0, stream=None):
+                                   v_block, scale: float = 0.0, out_nodes=None, out_suffix=None,
+                                   dev_status=None, workspace=None, stream=None):
     """The verification attention of a full-sequence bidirectional model that
     caches only its prefix (Fig. 3 caption, App. A.2): the block being decoded
     (node 0) and the trailing masked blocks attend to the whole true sequence,
-    every draft block to the prefix, the trailing blocks and itself.  Two calls
-    of spiffy_graph_attention on the tensor-core kernel:
-      nodes   context = [prefix ; suffix], blocks = the N node blocks;
-      suffix  one node whose block is the suffix, context = [prefix ; true block].
+    every draft block to the prefix, the trailing blocks and itself.
     q_nodes [B,N,L,Hq,d], q_suffix [B,S,Hq,d], k/v_prefix [B,P,Hkv,d], k/v_suffix
-    [B,S,Hkv,d], k/v_block [B,N,L,Hkv,d], all bf16, d = 128, S <= 1024.  The two
-    contexts are assembled with torch.cat here; a caller that keeps its cache as
-    [suffix | prefix | true block] can pass views to the two calls instead.
+    [B,S,Hkv,d], k/v_block [B,N,L,Hkv,d], all bf16, d = 128, S <= 1024.
     Returns (out_nodes [B,N,L,Hq,d], out_suffix [B,S,Hq,d])."""
-    B, S = q_suffix.shape[0], q_suffix.shape[1]
-    ctx_nodes_k = torch.cat([k_prefix, k_suffix], 1) if k_prefix is not None else k_suffix.contiguous()
-    ctx_nodes_v = torch.cat([v_prefix, v_suffix], 1) if v_prefix is not None else v_suffix.contiguous()
-    out_nodes = spiffy_graph_attention(q_nodes, ctx_nodes_k, ctx_nodes_v, k_block, v_block, scale=scale,
-                                       kernel=ATTN_TCGEN05, stream=stream)
-    true_k, true_v = k_block[:, 0], v_block[:, 0]
-    ctx_suffix_k = torch.cat([k_prefix, true_k], 1) if k_prefix is not None else true_k.contiguous()
-    ctx_suffix_v = torch.cat([v_prefix, true_v], 1) if v_prefix is not None else true_v.contiguous()
-    out_suffix = spiffy_graph_attention(q_suffix.unsqueeze(1).contiguous(), ctx_suffix_k, ctx_suffix_v,
-                                        k_suffix.unsqueeze(1).contiguous(), v_suffix.unsqueeze(1).contiguous(),
-                                        scale=scale, kernel=ATTN_TCGEN05, stream=stream)
-    return out_nodes, out_suffix.squeeze(1)
+    desc = attn_desc(q_nodes, k_prefix, k_block, scale, ATTN_TCGEN05)
+    S = int(q_suffix.shape[1])
+    if out_nodes is None:
+        out_nodes = torch.empty_like(q_nodes)
+    if out_suffix is None:
+        out_suffix = torch.empty_like(q_suffix)
+    need = int(lib().spiffy_full_sequence_attention_workspace(ctypes.byref(desc), S))
+    if need and workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q_nodes.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    dt = q_nodes.dtype
+    st = lib().spiffy_full_sequence_attention(
+        ctypes.byref(desc), S, _dev(q_nodes, "q_nodes"), _dev(q_suffix, "q_suffix", dt),
+        _dev(k_prefix, "k_prefix", dt), _dev(v_prefix, "v_prefix", dt), _dev(k_suffix, "k_suffix", dt),
+        _dev(v_suffix, "v_suffix", dt), _dev(k_block, "k_block", dt), _dev(v_block, "v_block", dt),
+        _dev(out_nodes, "out_nodes", dt), _dev(out_suffix, "out_suffix", dt),
+        _dev(dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"), ws_bytes, _stream(stream))
+    _check(st, "spiffy_full_sequence_attention")
+    return out_nodes, out_suffix
 
 
 @dataclass

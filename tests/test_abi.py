@@ -229,3 +229,23 @@ def test_binding_refuses_cpu_tensors():
     tok = torch.zeros(1, 1, 4, dtype=torch.int32)
     with pytest.raises(ValueError):
         spiffy.spiffy_unmask_decide(t, tok, 7, spiffy.RULE_TOPS)
+
+
+def test_full_sequence_attention_rejects_bad_arguments(lib):
+    fake = ctypes.c_void_p(0x1000)
+    good = spiffy.AttnDesc(1, 4, 32, 64, 8, 2, 128, spiffy.BF16, 0.0, spiffy.ATTN_TCGEN05)
+
+    def call(d, S=32, q_suffix=fake, k_prefix=fake, out_suffix=fake, k_block=fake):
+        return lib.spiffy_full_sequence_attention(ctypes.byref(d), S, fake, q_suffix, k_prefix, fake, fake, fake,
+                                                  k_block, fake, fake, out_suffix, None, None, 0, None)
+
+    assert call(good, q_suffix=None) == spiffy.EINVAL
+    assert call(good, out_suffix=None) == spiffy.EINVAL
+    assert call(good, k_prefix=None) == spiffy.EINVAL          # P > 0 needs a prefix
+    assert call(good, k_block=ctypes.c_void_p(0x1008)) == spiffy.EINVAL
+    assert call(good, S=-1) == spiffy.EINVAL
+    assert call(good, S=1025) == spiffy.EUNSUPPORTED
+    # the tensor-core kernel only: bf16, head dimension 128
+    assert call(spiffy.AttnDesc(1, 4, 32, 64, 8, 2, 128, spiffy.F32, 0.0, spiffy.ATTN_AUTO)) == spiffy.EUNSUPPORTED
+    assert call(spiffy.AttnDesc(1, 4, 32, 64, 8, 2, 64, spiffy.BF16, 0.0, spiffy.ATTN_AUTO)) == spiffy.EUNSUPPORTED
+    assert lib.spiffy_full_sequence_attention_workspace(ctypes.byref(good), 2000) == 0
