@@ -11,10 +11,10 @@ acceptance walk (step 5).  The metric is verify steps per second.
 `value`   : inputs resident in HBM, K steps replayed from a CUDA graph that
             rotates over several distinct input sets (together larger than
             L2), timed with CUDA events on the launching stream.
-`e2e`     : the same step driven from pinned host memory through
-            VerifyStep.run_host (host-to-device copies of everything the step
-            reads -- of the logits, the rows of still-masked positions -- and
-            the device-to-host read of the verdict inside the timed region).
+`e2e`     : the same step from pinned host memory through ONE C-ABI call,
+            spiffy_verify_step_host (host-to-device copies of everything the
+            step reads -- of the logits, the rows of still-masked positions --
+            and the device-to-host read of the verdict inside the timed region).
 `roofline`: the kernel with the largest share of a step (the attention kernel)
             against the roof that binds it at this shape, timed alone by
             replaying its call over the same rotation of input sets; the

@@ -29,6 +29,8 @@
  *                            logits are reduced on the tensor cores, never stored;
  *   spiffy_draft_blocks      drafting and pruning (Sec. 4.4.2, Sec. 4.4.4): the
  *                            draft blocks and parent lists of the next step;
+ *   spiffy_verify_step_host  one whole step (attention of one layer, steps 1-5)
+ *                            from tensors in host memory, copies included;
  *   spiffy_stage_masked_rows, spiffy_unmask_decide_static
  *                            helpers without a counterpart in the paper: staging
  *                            of logits from pinned host memory, and the decision
@@ -428,6 +430,55 @@ spiffy_status spiffy_decide_walk_lazy(const spiffy_decide_desc* desc, const void
                                       int32_t* n_accepted, int32_t* path, int32_t* next_block,
                                       int32_t* walk_status, void* workspace,
                                       size_t workspace_bytes, void* cuda_stream);
+
+/* ------------------------------------------------------------------------- */
+/* One whole verification step from HOST memory                                */
+/* ------------------------------------------------------------------------- */
+/*
+ * For a caller whose tensors are in host memory (the paper has no counterpart:
+ * its tensors never leave the device): copies the inputs of one verification
+ * step to the device, runs spiffy_graph_attention (one layer; Sec. 4.3) and
+ * spiffy_decide_walk (Algorithm 1, steps 1-5) on them, copies the verdict back
+ * and returns when it has arrived (the call synchronises `cuda_stream`).
+ *
+ * All tensor arguments are HOST pointers with the layouts of the component
+ * calls.  Pinned memory (cudaHostAlloc / cudaHostRegister) makes the copies
+ * asynchronous and lets one kernel read, of the logits, only the rows of
+ * still-masked positions -- the only ones the decision reads -- over the bus;
+ * pageable memory works too, through the runtime's staging, with all rows
+ * copied.  Everything but the logits travels on a helper stream of the library
+ * (created at the first call on a device) at the same time.
+ *
+ *   desc->attn, desc->decide   descriptors of the two component calls; batch,
+ *                    n_nodes and block_len must agree, block_len <= 64
+ *   desc->parent_cap entries per sequence in parent_idx
+ *   q .. parent_idx  inputs (k_prefix, v_prefix may be NULL when prefix_len == 0)
+ *   accepted_node [B], n_accepted [B], path [B][N], next_block [B][L]   the verdict
+ *   status [1 + 2B]  device status words: [0] attention, [1 .. B] decision per
+ *                    sequence, [1+B .. 2B] walk per sequence (SPIFFY_DEV_* bits)
+ *   device_workspace DEVICE memory, 256-byte aligned, of
+ *                    spiffy_verify_step_host_workspace(desc) bytes: staging copies
+ *                    of every input, the attention output and the decision's
+ *                    per-node results (which stay there), the kernels' scratch
+ * Calls sharing a workspace, or made from several threads on one device, must
+ * not overlap (the helper stream is shared).
+ */
+typedef struct {
+  spiffy_attn_desc attn;
+  spiffy_decide_desc decide;
+  int32_t parent_cap;
+} spiffy_step_desc;
+
+size_t spiffy_verify_step_host_workspace(const spiffy_step_desc* desc);
+spiffy_status spiffy_verify_step_host(const spiffy_step_desc* desc, const void* q,
+                                      const void* k_prefix, const void* v_prefix,
+                                      const void* k_block, const void* v_block,
+                                      const void* logits, const int32_t* block_tokens,
+                                      const int32_t* parent_off, const int32_t* parent_idx,
+                                      int32_t* accepted_node, int32_t* n_accepted, int32_t* path,
+                                      int32_t* next_block, int32_t* status,
+                                      void* device_workspace, size_t workspace_bytes,
+                                      void* cuda_stream);
 
 /*
  * Staging helper for callers whose logits sit in pinned host memory (the paper

@@ -50,6 +50,10 @@ class DecideDesc(ctypes.Structure):
                 ("top_s", ctypes.c_int32), ("threshold", ctypes.c_float)]
 
 
+class StepDesc(ctypes.Structure):
+    _fields_ = [("attn", AttnDesc), ("decide", DecideDesc), ("parent_cap", ctypes.c_int32)]
+
+
 class SampleDesc(ctypes.Structure):
     _fields_ = [("temperature", ctypes.c_float), ("reserved", ctypes.c_uint32), ("seed", ctypes.c_uint64)]
 
@@ -111,6 +115,10 @@ def lib() -> ctypes.CDLL:
         L.spiffy_lmhead_decide_workspace.argtypes = [ctypes.POINTER(DecideDesc), i32]
         L.spiffy_lmhead_decide.restype = ctypes.c_int
         L.spiffy_lmhead_decide.argtypes = [ctypes.POINTER(DecideDesc), i32] + [vp] * 9 + [sz, vp]
+        L.spiffy_verify_step_host_workspace.restype = sz
+        L.spiffy_verify_step_host_workspace.argtypes = [ctypes.POINTER(StepDesc)]
+        L.spiffy_verify_step_host.restype = ctypes.c_int
+        L.spiffy_verify_step_host.argtypes = [ctypes.POINTER(StepDesc)] + [vp] * 15 + [sz, vp]
         L.spiffy_status_string.restype = ctypes.c_char_p
         L.spiffy_status_string.argtypes = [ctypes.c_int]
         L.spiffy_launch_count.restype = ctypes.c_uint64
@@ -475,6 +483,48 @@ def spiffy_stage_masked_rows(src_logits, dst_logits, tokens, mask_token_id: int,
                                         tokens.numel(), _stream(stream))
     _check(st, "spiffy_stage_masked_rows")
     return dst_logits
+
+
+def _host(t: Optional[torch.Tensor], name: str, dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    if t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous host tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def step_desc(q, k_prefix, k_block, logits, block_tokens, parent_idx, mask_token_id, rule, top_s=1,
+              threshold=0.9, scale=0.0, kernel=ATTN_AUTO) -> StepDesc:
+    return StepDesc(attn_desc(q, k_prefix, k_block, scale, kernel),
+                    decide_desc(logits, block_tokens, mask_token_id, rule, top_s, threshold),
+                    int(parent_idx.shape[1]))
+
+
+def spiffy_verify_step_host_workspace(desc: StepDesc) -> int:
+    return int(lib().spiffy_verify_step_host_workspace(ctypes.byref(desc)))
+
+
+def spiffy_verify_step_host(desc: StepDesc, q, k_prefix, v_prefix, k_block, v_block, logits, block_tokens,
+                            parent_off, parent_idx, accepted_node, n_accepted, path, next_block, status,
+                            device_workspace, stream=None):
+    """One whole verification step from HOST tensors (pinned for speed): the
+    inputs are copied in, attention + decision + walk run on the device, and the
+    verdict (accepted_node [B], n_accepted [B], path [B,N], next_block [B,L], all
+    int32 host tensors, plus status [1+2B]) is back when the call returns."""
+    i32 = torch.int32
+    dt = q.dtype
+    st = lib().spiffy_verify_step_host(
+        ctypes.byref(desc), _host(q, "q"), _host(k_prefix, "k_prefix", dt), _host(v_prefix, "v_prefix", dt),
+        _host(k_block, "k_block", dt), _host(v_block, "v_block", dt), _host(logits, "logits"),
+        _host(block_tokens, "block_tokens", i32), _host(parent_off, "parent_off", i32),
+        _host(parent_idx, "parent_idx", i32), _host(accepted_node, "accepted_node", i32),
+        _host(n_accepted, "n_accepted", i32), _host(path, "path", i32), _host(next_block, "next_block", i32),
+        _host(status, "status", i32), _dev(device_workspace, "device_workspace"),
+        device_workspace.numel() * device_workspace.element_size(), _stream(stream))
+    _check(st, "spiffy_verify_step_host")
+    return accepted_node, n_accepted, path, next_block, status
 
 
 @dataclass

@@ -4,8 +4,9 @@ copies); all arithmetic happens inside ``libspiffy.so``.
 
 ``VerifyStep`` owns preallocated outputs and workspaces so that a step issues
 no allocation and can be captured into a CUDA graph.  ``run`` takes device
-tensors; ``run_host`` takes pinned host tensors, copies them in, runs the step
-and copies the verdict back -- the end-to-end call.
+tensors; ``run_host`` takes host tensors (pinned for speed) and makes the whole
+step one C-ABI call that copies them in, runs the step and brings the verdict
+back -- the end-to-end call.
 """
 from __future__ import annotations
 
@@ -85,16 +86,11 @@ class VerifyStep:
             torch.empty((B, N), dtype=torch.int32, device=dev),
             torch.empty((B, L), dtype=torch.int32, device=dev),
             torch.zeros((B,), dtype=torch.int32, device=dev))
-        # the verdict a caller reads back: accepted node, hop count, next block
-        pin = dev.type == "cuda"
-        host = lambda t: torch.empty_like(t, device="cpu").pin_memory() if pin else None
-        self.verdict_host = (host(self.walk.accepted_node), host(self.walk.n_accepted),
-                             host(self.walk.next_block))
-        self.staging = None
+        self.host_ws = None
+        self.host_desc = None
+        self.host_verdict = None
         self.lazy_ws = None
         self.sampled_ws = None
-        self.copy_stream = None
-        self.copy_events = None
 
     # the three calls of one step, asynchronous on the current stream
     def attention(self, x: StepInputs):
@@ -146,50 +142,38 @@ class VerifyStep:
         self.attention(x)
         return self.decide_accept(x)
 
-    @staticmethod
-    def _masked_row_runs(host: StepInputs, mask_id: int):
-        """[start, stop) runs of logit rows whose position is still masked: the
-        only rows the decision step reads (Algorithm 1 ranks masked positions)."""
-        m = (host.block_tokens.reshape(-1) == mask_id).to(torch.int8)
-        edges = torch.diff(m, prepend=m.new_zeros(1), append=m.new_zeros(1)).nonzero().reshape(-1).tolist()
-        return list(zip(edges[0::2], edges[1::2]))
-
     def run_host(self, host: StepInputs):
-        """End to end from pinned host memory: copy the step's inputs in, run
-        it, read the verdict (accepted node, hop count, next block) back.  Of
-        the logits only the rows of still-masked positions cross the bus
-        (spiffy_stage_masked_rows reads them from the pinned buffer); the
-        staging rows of unmasked positions keep whatever they held and no
-        kernel reads them."""
-        if self.staging is None:
-            self.staging = StepInputs(*[torch.empty_like(t, device=self.device) for t in host.tensors()])
-        main = torch.cuda.current_stream()
-        if self.copy_stream is None:
-            self.copy_stream = torch.cuda.Stream(self.device)
-            self.copy_events = (torch.cuda.Event(), torch.cuda.Event())
-        # the small tensors go through the copy engine on a side stream while one kernel pulls
-        # the masked logits rows over the bus; both start once the staging buffers are free
-        self.copy_events[0].record(main)
-        self.copy_stream.wait_event(self.copy_events[0])
-        with torch.cuda.stream(self.copy_stream):
-            for dst, src in zip(self.staging.tensors(), host.tensors()):
-                if src is not host.logits:
-                    dst.copy_(src, non_blocking=True)
-            self.copy_events[1].record(self.copy_stream)
-        spiffy.spiffy_stage_masked_rows(host.logits, self.staging.logits, host.block_tokens, self.cfg.mask_id)
-        main.wait_event(self.copy_events[1])
-        w = self.run(self.staging)
-        for dst, src in zip(self.verdict_host, (w.accepted_node, w.n_accepted, w.next_block)):
-            dst.copy_(src, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
-        return self.verdict_host
+        """End to end from pinned host memory through the C ABI's host-buffer
+        entry (spiffy_verify_step_host): the step's inputs are copied in -- of
+        the logits only the rows of still-masked positions cross the bus --, the
+        step runs, and the verdict (accepted node, hop count, path, next block)
+        is in host memory when the call returns."""
+        c = self.cfg
+        B, N, L = c.batch, c.n_nodes, c.block_len
+        if self.host_ws is None:
+            self.host_desc = spiffy.step_desc(host.q, host.k_prefix, host.k_block, host.logits, host.block_tokens,
+                                              host.parent_idx, c.mask_id, c.rule, c.top_s, c.threshold,
+                                              kernel=self.attn_kernel)
+            need = spiffy.spiffy_verify_step_host_workspace(self.host_desc)
+            self.host_ws = torch.empty((need + 256,), dtype=torch.uint8, device=self.device)
+            off = (-self.host_ws.data_ptr()) % 256
+            self.host_ws = self.host_ws[off:off + need]
+            pin = lambda *shape: torch.empty(shape, dtype=torch.int32).pin_memory()
+            self.host_verdict = (pin(B), pin(B), pin(B, N), pin(B, L), pin(1 + 2 * B))
+        kp = host.k_prefix if c.prefix_len else None
+        vp = host.v_prefix if c.prefix_len else None
+        return spiffy.spiffy_verify_step_host(self.host_desc, host.q, kp, vp, host.k_block, host.v_block,
+                                              host.logits, host.block_tokens, host.parent_off, host.parent_idx,
+                                              *self.host_verdict, self.host_ws)
 
     def h2d_bytes(self, host: StepInputs) -> int:
         """Bytes ``run_host`` copies to the device for this input."""
-        rows = sum(b - a for a, b in self._masked_row_runs(host, self.cfg.mask_id))
+        rows = int((host.block_tokens == self.cfg.mask_id).sum())
         V = host.logits.shape[-1]
         return host.nbytes() - host.logits.numel() * host.logits.element_size() \
             + rows * V * host.logits.element_size()
 
     def d2h_bytes(self) -> int:
-        return sum(t.numel() * t.element_size() for t in self.verdict_host)
+        c = self.cfg
+        B, N, L = c.batch, c.n_nodes, c.block_len
+        return 4 * (B + B + B * N + B * L + 1 + 2 * B)

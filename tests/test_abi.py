@@ -249,3 +249,27 @@ def test_full_sequence_attention_rejects_bad_arguments(lib):
     assert call(spiffy.AttnDesc(1, 4, 32, 64, 8, 2, 128, spiffy.F32, 0.0, spiffy.ATTN_AUTO)) == spiffy.EUNSUPPORTED
     assert call(spiffy.AttnDesc(1, 4, 32, 64, 8, 2, 64, spiffy.BF16, 0.0, spiffy.ATTN_AUTO)) == spiffy.EUNSUPPORTED
     assert lib.spiffy_full_sequence_attention_workspace(ctypes.byref(good), 2000) == 0
+
+
+def test_host_step_rejects_bad_arguments(lib):
+    fake = ctypes.c_void_p(0x1000)
+    attn = spiffy.AttnDesc(1, 4, 8, 16, 4, 4, 64, spiffy.F32, 0.0, spiffy.ATTN_AUTO)
+    dec = spiffy.DecideDesc(1, 4, 8, 1024, spiffy.F32, 1024, 1023, spiffy.RULE_TOPS, 1, 0.9)
+    good = spiffy.StepDesc(attn, dec, 4)
+    need = lib.spiffy_verify_step_host_workspace(ctypes.byref(good))
+    # staging of every input, the attention output, the decision's results and scratch
+    assert need > 2 * 1 * 4 * 8 * 4 * 64 * 4 + 4 * 8 * 1024 * 4
+
+    def call(d, q=fake, out=fake, ws=ctypes.c_void_p(0x10000), ws_bytes=1 << 30):
+        return lib.spiffy_verify_step_host(ctypes.byref(d), q, fake, fake, fake, fake, fake, fake, fake, fake,
+                                           out, fake, fake, fake, fake, ws, ws_bytes, None)
+
+    assert call(good, q=None) == spiffy.EINVAL
+    assert call(good, out=None) == spiffy.EINVAL
+    assert call(good, ws=None) == spiffy.EWORKSPACE
+    assert call(good, ws_bytes=need - 1) == spiffy.EWORKSPACE
+    assert call(good, ws=ctypes.c_void_p(0x10010)) == spiffy.EWORKSPACE   # 256-byte alignment
+    mismatch = spiffy.StepDesc(attn, spiffy.DecideDesc(1, 5, 8, 1024, spiffy.F32, 1024, 1023, spiffy.RULE_TOPS, 1, 0.9), 4)
+    assert call(mismatch) == spiffy.EINVAL
+    assert lib.spiffy_verify_step_host_workspace(ctypes.byref(mismatch)) == 0
+    assert call(spiffy.StepDesc(attn, dec, 0)) == spiffy.EINVAL
