@@ -60,6 +60,10 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-composite", action="store_true", help="skip the whole-model (one attention call per layer) step")
     ap.add_argument("--no-other-shapes", action="store_true", help="skip the timing of the other configurations")
+    ap.add_argument("--profile", action="store_true",
+                    help="bounded run for a profiler: one timed region of exactly the asked steps (rounded up to "
+                         "whole rotations), no per-call timing repeats, no whole-model step, other shapes, "
+                         "end-to-end or CPU-baseline legs")
     ap.add_argument("--no-early-dependents", action="store_true",
                     help="whole-model step without SPIFFY_ATTN_EARLY_DEPENDENTS on the layers' attention calls")
     ap.add_argument("--part", default="step", choices=["step", "attention", "full_sequence", "decide", "decide_walk", "decide_walk_lazy", "decide_sampled", "lmhead", "draft"],
@@ -619,7 +623,7 @@ def main():
     stream = torch.cuda.Stream()
     sampler = ClockSampler(local)
     with torch.cuda.stream(stream):
-        timer = GraphTimer(stream)
+        timer = GraphTimer(stream, repeats=1, min_region_s=0.0) if args.profile else GraphTimer(stream)
         # eager warm-up (also loads the kernels), then capture one rotation over the input sets
         for i in range(max(3, min(args.warmup, 2 * N_SETS))):
             step.run(sets[i % N_SETS])
@@ -656,7 +660,7 @@ def main():
         # one verification step of a whole model: the attention runs once per layer, each layer
         # on its own q/K/V (32 layers x 16.8 MB: L2-cold by construction), then one decision + walk
         composite = None
-        if args.config in (2, 3, 4, 5) and not args.no_composite:
+        if args.config in (2, 3, 4, 5) and not args.no_composite and not args.profile:
             layers = 28 if args.config == 3 else 32
             layer_sets = device_attention_inputs(cfg, layers, 7)
             # in a layer loop the next kernel may begin its set-up while this one drains
@@ -690,11 +694,11 @@ def main():
             del layer_sets, layer_fns, cg, ag
 
         shapes = None
-        if rank == 0 and world == 1 and args.config == 2 and not args.no_other_shapes:
+        if rank == 0 and world == 1 and args.config == 2 and not args.no_other_shapes and not args.profile:
             shapes = other_shapes(timer, peaks)
 
         # end to end from pinned host memory
-        n_e2e = max(5, min(50, steps))
+        n_e2e = 1 if args.profile else max(5, min(50, steps))
         for _ in range(3):
             step.run_host(host0)
         torch.cuda.synchronize()
@@ -781,7 +785,7 @@ def main():
         line["composite_model_step"] = composite
     if shapes is not None:
         line["other_shapes"] = shapes
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.profile:
         import oracle
         sec, what = oracle_step_time(cfg, work[0], 80)  # about ten seconds of CPU work
         line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": oracle.max_threads(),
