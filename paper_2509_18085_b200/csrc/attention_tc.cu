@@ -214,7 +214,11 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
   uint64_t* v_empty = v_full + VS;
   uint64_t* s_full = v_empty + VS;   // [2]
   uint64_t* p_ready = s_full + 2;    // [2]
-  uint64_t* pv_done = p_ready + 2;   // [2]: NQ = 2 one per warpgroup; NQ = 1 only the first
+  // P V products done.  NQ = 2: one barrier per warpgroup (a thread is never more than one tile
+  // ahead of its products).  NQ = 1: one per parity of the key tile: S is double buffered there, a
+  // softmax thread may be two tiles ahead of the products, and the phase parity of ONE barrier
+  // cannot tell "tile j - 2 still running" from "tile j - 1 done".
+  uint64_t* pv_done = p_ready + 2;   // [2]
   uint64_t* xchg_ready = pv_done + 2;  // pair: the peer's Q tile and first K stage may be overwritten
   uint64_t* xchg_full = xchg_ready + 1;  // pair: the peer's partial has arrived here
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + SM::tmem);
@@ -384,7 +388,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
           umma_ts_k64(tmem + kColO, a, vj, hi, idesc_o, j > 0 ? 1u : 0u);
           umma_ts_k64(tmem + kColO + HD, a + 64u, vj + 4u * 128u, hi, idesc_o, j > 0 ? 1u : 0u);
           umma_commit(v_empty + j % VS);
-          umma_commit(pv_done);
+          umma_commit(pv_done + (j & 1));
           if (j + 2 < T) s_tile(j + 2);
         }
       } else {
@@ -429,12 +433,16 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     bool ok = true;
     // this thread's accumulator: NQ = 1 columns half wg of every tile, NQ = 2 all of M-tile wg
     const uint32_t col_o = kColO + (uint32_t)wg * HD;
-    uint64_t* my_pv_done = NQ == 1 ? pv_done : pv_done + wg;
+    // every product into this thread's accumulator up to key tile j has completed
+    auto wait_pv = [&](int j) -> bool {
+      uint64_t* bar = NQ == 1 ? pv_done + (j & 1) : pv_done + wg;
+      const uint32_t parity = NQ == 1 ? (uint32_t)(j >> 1) & 1u : (uint32_t)j & 1u;
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, p.spin_limit));
+    };
 
     // O *= corr once the products that still write to it have completed
     auto rescale_o = [&](int j, float corr) -> bool {
-      if (!__all_sync(0xffffffffu, mbar_wait(my_pv_done, (uint32_t)(j - 1) & 1u, abort_flag, p.spin_limit)))
-        return false;
+      if (!wait_pv(j - 1)) return false;
       tc_fence_after_sync();
 #pragma unroll
       for (int c0 = 0; c0 < HD; c0 += 32) {
@@ -542,8 +550,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     }
     // ------------------------------------------------------------ epilogue --
     // every product into this thread's accumulator has completed
-    if (ok)
-      ok = __all_sync(0xffffffffu, mbar_wait(my_pv_done, (uint32_t)(T - 1) & 1u, abort_flag, p.spin_limit));
+    if (ok) ok = wait_pv(T - 1);
     __nv_bfloat16* dst =
         p.out + (((int64_t)b * p.NL + nl) * p.Hq + (int64_t)g * p.group + hh) * HD;
     if constexpr (NQ == 2) {
