@@ -271,16 +271,29 @@ spiffy_status spiffy_unmask_decide_static(const spiffy_decide_desc* desc,
 /*
  * The decision step at sampling temperature T > 0 (Sec. 5.3, "Effect of Temperature", runs Spiffy at
  * T > 0; the sampler itself is not given in the paper and is fixed here).
- * Per still-masked position the token is drawn from softmax(x / T) as
- *   top_tok = argmax_v (x_v / T + g_v),  g_v = -ln(-ln u_v)      (Gumbel-max)
- * and conf is its probability softmax(x / T)[top_tok]; the unmasking rule then
- * runs on conf exactly as in spiffy_unmask_decide, and every other argument,
- * layout and status bit is that call's.
- * The uniforms u_v come from the counter-based generator Philox4x32-10
- * (Salmon, Moraes, Dror, Shaw, SC 2011):
- *   counter = (v / 4, position l, sequence b, number of still-masked positions
- *              of the node),  key = (seed & 0xffffffff, seed >> 32),
- *   u_v = (output word v % 4 + 0.5) / 2^32.
+ * Per still-masked position the token is drawn from softmax(z), z = x / T, in
+ * two levels over vocabulary slices of W = spiffy_sampled_slice_width(desc)
+ * consecutive entries (slice s = entries s W ... s W + W - 1):
+ *   1. the slice  s* = argmax_s (ln Z_s + g_s),  Z_s = sum over the slice of
+ *      exp(z_v),  g_s = -ln(-ln u_s)   (Gumbel-max on the slices' weights; ties
+ *      to the lower slice, a slice without weight never wins);
+ *   2. top_tok = the first entry v of slice s*, ascending, whose running sum
+ *      sum_{w <= v in s*} exp(z_w) reaches u' Z_s*   (inversion inside the slice);
+ * conf is its probability softmax(z)[top_tok]; the unmasking rule then runs on
+ * conf exactly as in spiffy_unmask_decide, and every other argument, layout and
+ * status bit is that call's.  One pass over the logits plus one slice per row:
+ * the cost of the greedy decision, not of V random numbers per row.
+ * The uniforms come from the counter-based generator Philox4x32-10 (Salmon,
+ * Moraes, Dror, Shaw, SC 2011):
+ *   counter = (slice s, position l, sequence b, number of still-masked
+ *              positions of the node),  key = (seed & 0xffffffff, seed >> 32),
+ *   u_s = (output word 0 + 0.5) / 2^32,  u' = (output word 1 + 0.5) / 2^32 of
+ *   the chosen slice's counter.
+ * W is the width of the slices the kernels reduce in one piece: the vocabulary
+ * cut into the fewest equal slices of at most 8192 (bf16) or 4096 (fp32)
+ * entries, rounded up to a multiple of 8 (bf16) or 4 (fp32); 0 for a bad
+ * descriptor.  It is part of the sampler's definition: another W gives other
+ * (equally distributed) tokens for the same seed.
  * The noise depends on the state of the block, not on the node's index: a
  * draft block and the true block that equals it draw the same tokens, which is
  * what the losslessness argument of App. A needs.  A caller that wants fresh
@@ -294,6 +307,7 @@ typedef struct {
 } spiffy_sample_desc;
 
 size_t spiffy_unmask_decide_sampled_workspace(const spiffy_decide_desc* desc);
+int64_t spiffy_sampled_slice_width(const spiffy_decide_desc* desc);
 spiffy_status spiffy_unmask_decide_sampled(const spiffy_decide_desc* desc,
                                            const spiffy_sample_desc* sample, const void* logits,
                                            const int32_t* block_tokens, float* conf,

@@ -278,6 +278,13 @@ size_t spiffy_unmask_decide_sampled_workspace(const spiffy_decide_desc* desc) {
   return decide_sampled_workspace_bytes(*desc);
 }
 
+int64_t spiffy_sampled_slice_width(const spiffy_decide_desc* desc) {
+  if (check_decide_desc(desc, true) != SPIFFY_OK) return 0;
+  int64_t chunk = 0;
+  decide_splits(*desc, &chunk);
+  return chunk;
+}
+
 spiffy_status spiffy_unmask_decide_sampled(const spiffy_decide_desc* desc,
                                            const spiffy_sample_desc* sample, const void* logits,
                                            const int32_t* block_tokens, float* conf,

@@ -142,10 +142,13 @@ struct Elem<float> {
 // slice is at most kReduceThreads * kUnroll vectors, so that every thread holds
 // its whole share in registers: all loads go out at once, the slice maximum is
 // found first and the exponentials are then taken against it directly.  All
-// threads of the CTA call it together; thread 0 stores the result.
+// threads of the CTA call it together; thread 0 stores the result.  `k` is
+// log2(e) for the plain softmax; the sampled decision passes log2(e) / T and
+// gets the sum of exp((x - maximum) / T).
 template <typename T>
 __device__ __forceinline__ void reduce_slice(const T* __restrict__ base, int V, int64_t chunk,
-                                             int split, Partial* __restrict__ out) {
+                                             int split, Partial* __restrict__ out,
+                                             const float k = kLog2e) {
   const int64_t begin = (int64_t)split * chunk;
   const int64_t end = min((int64_t)V, begin + chunk);
   constexpr int EPV = Elem<T>::kPerVec;
@@ -180,8 +183,8 @@ __device__ __forceinline__ void reduce_slice(const T* __restrict__ base, int V, 
 #pragma unroll
   for (int w = 1; w < kReduceThreads / 32; ++w) m = fmaxf(m, warp_m[w]);
   // 3. sum of exp(x - m) and the lowest index that attains m
-  const float ml = (m == -INFINITY) ? 0.f : m * kLog2e;  // an all -inf slice sums to 0
-  const uint64_t k2 = pack2(kLog2e, kLog2e), nml2 = pack2(-ml, -ml);
+  const float ml = (m == -INFINITY) ? 0.f : m * k;  // an all -inf slice sums to 0
+  const uint64_t k2 = pack2(k, k), nml2 = pack2(-ml, -ml);
   uint64_t acc = pack2(0.f, 0.f);
   int idx = 0x7fffffff;
 #pragma unroll
@@ -200,7 +203,7 @@ __device__ __forceinline__ void reduce_slice(const T* __restrict__ base, int V, 
     int tidx = 0x7fffffff;
 #pragma unroll
     for (int e = EPV - 1; e >= 0; --e) {
-      s += ex2(fmaf(tail[e], kLog2e, -ml));  // -inf beyond the tail: adds 0
+      s += ex2(fmaf(tail[e], k, -ml));  // -inf beyond the tail: adds 0
       if (e < ntail && tail[e] == m) tidx = (int)begin + nvec * EPV + e;
     }
     idx = min(idx, tidx);

@@ -108,6 +108,8 @@ def lib() -> ctypes.CDLL:
         L.spiffy_stage_masked_rows.argtypes = [vp, vp, ctypes.c_int64, vp, i32, ctypes.c_int64, vp]
         L.spiffy_unmask_decide_sampled_workspace.restype = sz
         L.spiffy_unmask_decide_sampled_workspace.argtypes = [ctypes.POINTER(DecideDesc)]
+        L.spiffy_sampled_slice_width.restype = ctypes.c_int64
+        L.spiffy_sampled_slice_width.argtypes = [ctypes.POINTER(DecideDesc)]
         L.spiffy_unmask_decide_sampled.restype = ctypes.c_int
         L.spiffy_unmask_decide_sampled.argtypes = [ctypes.POINTER(DecideDesc), ctypes.POINTER(SampleDesc)] + \
             [vp] * 8 + [sz, vp]
@@ -296,8 +298,9 @@ def spiffy_unmask_decide_sampled(logits, block_tokens, mask_token_id: int, rule:
                                  seed: int, top_s: int = 1, threshold: float = 0.9,
                                  out: Optional[Decision] = None, workspace=None, stream=None) -> Decision:
     """Steps 1-4 of Algorithm 1 at sampling temperature T > 0: tokens drawn from
-    softmax(x / T) by Gumbel-max with Philox4x32-10 noise that follows the
-    block's state (sequence, position, vocabulary entry, masked count), never
+    softmax(x / T) in two levels (Gumbel-max over vocabulary slices, inversion
+    of the running sum inside the chosen slice) with Philox4x32-10 noise that
+    follows the block's state (sequence, position, slice, masked count), never
     the node's index; conf is the drawn token's probability."""
     desc = decide_desc(logits, block_tokens, mask_token_id, rule, top_s, threshold)
     sample = SampleDesc(float(temperature), 0, int(seed) & 0xFFFFFFFFFFFFFFFF)
@@ -318,6 +321,11 @@ def spiffy_unmask_decide_sampled(logits, block_tokens, mask_token_id: int, rule:
         workspace.numel() * workspace.element_size(), _stream(stream))
     _check(st, "spiffy_unmask_decide_sampled")
     return out
+
+
+def spiffy_sampled_slice_width(desc: DecideDesc) -> int:
+    """Width of the vocabulary slices of the sampled decision's two-level draw."""
+    return int(lib().spiffy_sampled_slice_width(ctypes.byref(desc)))
 
 
 def spiffy_lmhead_decide(hidden_states, weight, block_tokens, mask_token_id: int, rule: int,

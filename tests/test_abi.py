@@ -27,7 +27,7 @@ def declared_functions():
 def test_every_declared_symbol_is_exported(lib):
     names = declared_functions()
     assert {"spiffy_graph_attention", "spiffy_unmask_decide", "spiffy_accept_walk"} <= set(names)
-    assert len(names) >= 19
+    assert len(names) >= 20
     for name in names:
         assert getattr(lib, name) is not None
         # the binding gives every entry point a prototype: nothing is called through ctypes' defaults
@@ -162,7 +162,16 @@ def test_sampled_decide_rejects_bad_arguments(lib):
     fake = ctypes.c_void_p(0x1000)
     good = spiffy.DecideDesc(1, 4, 8, 1024, spiffy.BF16, 1024, 1023, spiffy.RULE_TOPS, 1, 0.9)
     need = lib.spiffy_unmask_decide_sampled_workspace(ctypes.byref(good))
-    assert need == 2 * lib.spiffy_unmask_decide_workspace(ctypes.byref(good))  # 32-byte partial results
+    # the greedy call's partial results (rounded up to 256 bytes) and one arrival counter per node
+    greedy = lib.spiffy_unmask_decide_workspace(ctypes.byref(good))
+    assert need == (greedy + 255) // 256 * 256 + 4 * 4
+    # slice width: the fewest equal slices of at most 8192 bf16 / 4096 fp32 entries, whole 16-byte vectors
+    width = lambda v, dt: lib.spiffy_sampled_slice_width(ctypes.byref(
+        spiffy.DecideDesc(1, 4, 8, v, dt, v, v - 1, spiffy.RULE_TOPS, 1, 0.9)))
+    assert width(1024, spiffy.BF16) == 1024 and width(8192, spiffy.BF16) == 8192
+    assert width(126464, spiffy.BF16) == 7904 and width(8200, spiffy.BF16) == 4104
+    assert width(4100, spiffy.F32) == 2052 and width(36, spiffy.F32) == 36
+    assert width(0, spiffy.BF16) == 0
 
     def call(temperature=1.0, sample=True, logits=fake, ws=fake, ws_bytes=1 << 30, d=good):
         s = spiffy.SampleDesc(temperature, 0, 42)
