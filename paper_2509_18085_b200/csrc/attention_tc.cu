@@ -282,7 +282,7 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     prefetch_tensormap(p.TP1 > 0 ? &tm_kp : (p.TP > 0 ? &tm_kp2 : &tm_kb));
     mbar_init(q_full, 1);
     for (int i = 0; i < KS; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_ready + i, NQ == 1 ? 256 : 128); }
+    for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_ready + i, NQ == 1 ? 8 : 4); }  // one arrival per softmax warp
     mbar_init(pv_done, 1);
     mbar_init(pv_done + 1, 1);
     mbar_init(xchg_ready, 1);
@@ -506,7 +506,8 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         tmem_st_x32(tmem_addr(tmem, lane_base, col_s), pk);
         tmem_wait_st();
         tc_fence_before_sync();
-        mbar_arrive(p_ready + bi);
+        __syncwarp();  // every lane's P is in tensor memory: one arrival speaks for the warp
+        if (lane == 0) mbar_arrive(p_ready + bi);
       }
     } else {
       for (int j = 0; j < T; ++j) {
@@ -545,7 +546,8 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         tmem_st_x64(tmem_addr(tmem, lane_base, col_s), pk);
         tmem_wait_st();
         tc_fence_before_sync();
-        mbar_arrive(p_ready + wg);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(p_ready + wg);
       }
     }
     // ------------------------------------------------------------ epilogue --

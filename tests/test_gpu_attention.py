@@ -80,6 +80,26 @@ def test_odd_shapes(shape, dtype, kernel):
     assert np.max(np.abs(got - want)) <= G.TOL[dtype]
 
 
+@pytest.mark.parametrize("prefix_len,n_nodes,block_len", [
+    (384, 8, 32),   # 3 context tiles + 1 block tile: even, the two CTAs of a pair each finish half the columns
+    (512, 8, 32),   # 5 key tiles: odd, one CTA of the pair has a tile more
+    (640, 8, 32),   # 6
+    (300, 4, 32),   # 4, ragged context tile, one M-tile per head
+    (400, 6, 48),   # nodes of 48 positions: M-tiles with one and with two block-key tiles (odd and even in one launch)
+    (257, 3, 7),    # 4 tiles, a nearly empty M-tile
+])
+def test_cluster_pairs_with_even_and_odd_tile_counts(prefix_len, n_nodes, block_len):
+    """Few M-tiles (at most 74): the key tiles of each M-tile are split over the
+    two CTAs of a cluster, which merge through each other's shared memory."""
+    cfg = W.Config("pairs", dtype="bf16", vocab=16, rule=0, batch=1, n_nodes=n_nodes, block_len=block_len,
+                   prefix_len=prefix_len, n_q_heads=16, n_kv_heads=16, head_dim=128)
+    w = W.make(cfg, 31 + prefix_len, decision=False)
+    got = G.gpu_attention(w, spiffy.ATTN_TCGEN05)
+    want = oracle_attention(w)
+    assert np.max(np.abs(got - want)) <= G.TOL["bf16"]
+    assert np.sqrt(np.mean((got - want) ** 2)) < 2e-3
+
+
 @pytest.mark.parametrize("kernel", KERNELS)
 def test_custom_scale(kernel):
     cfg = W.config(2, n_nodes=2, prefix_len=200)
