@@ -140,16 +140,25 @@ decide_sampled_select_kernel(const T* __restrict__ logits, int64_t row_stride, i
                              int* __restrict__ node_count, float* __restrict__ conf_out,
                              int32_t* __restrict__ tok_out, uint64_t* __restrict__ bits_out,
                              int32_t* __restrict__ n_unmask_out, int32_t* __restrict__ dev_status) {
-#if __CUDA_ARCH__ >= 900
-  pdl_launch_dependents();
-  cudaGridDependencySynchronize();  // the reduce kernel's partials and cleared counters are visible
-#endif
   constexpr int EPV = Elem<T>::kPerVec;
   constexpr uint32_t NI = Elem<T>::kNegInf;
   const int row = blockIdx.x;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int node = row / L, l = row - node * L, b = node / N;
+  // The block's tokens were there before the reduce kernel started: they are read, and the
+  // node's masked positions counted, ahead of the wait for that kernel.
   const int32_t state = block_tokens[row];
+  int masked_count = 0;  // how far the node has been denoised: part of the noise's counter
+  if (warp == 0) {
+    const int32_t* st = block_tokens + (int64_t)node * L;
+    const bool m0 = lane < L && st[min(lane, L - 1)] == mask_id;
+    const bool m1 = lane + 32 < L && st[min(lane + 32, L - 1)] == mask_id;
+    masked_count = __popc(__ballot_sync(0xffffffffu, m0)) + __popc(__ballot_sync(0xffffffffu, m1));
+  }
+#if __CUDA_ARCH__ >= 900
+  pdl_launch_dependents();
+  cudaGridDependencySynchronize();  // the reduce kernel's partials and cleared counters are visible
+#endif
   const float k = inv_t * kLog2e;
   __shared__ SliceChoice choice;
   __shared__ double warp_total[kReduceThreads / 32];
@@ -158,13 +167,6 @@ decide_sampled_select_kernel(const T* __restrict__ logits, int64_t row_stride, i
   if (state == mask_id) {  // the whole CTA takes the same branch
     if (warp == 0) {
       // level 1: lanes over slices
-      int masked_count;  // how far the node has been denoised: part of the noise's counter
-      {
-        const int32_t* st = block_tokens + (int64_t)node * L;
-        const bool m0 = lane < L && st[min(lane, L - 1)] == mask_id;
-        const bool m1 = lane + 32 < L && st[min(lane + 32, L - 1)] == mask_id;
-        masked_count = __popc(__ballot_sync(0xffffffffu, m0)) + __popc(__ballot_sync(0xffffffffu, m1));
-      }
       const Philox rng{seed_lo, seed_hi, (uint32_t)l, (uint32_t)b, (uint32_t)masked_count};
       float rm = -INFINITY, rs = 0.f;      // row maximum of x and sum of exp((x - rm) / T)
       float best = -INFINITY, bm = 0.f, bz = 0.f;
