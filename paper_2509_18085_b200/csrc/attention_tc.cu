@@ -379,8 +379,12 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         s_tile(0);
         if (T > 1) s_tile(1);
         for (int j = 0; j < T && ok; ++j) {
-          if (!mbar_wait(p_ready + (j & 1), (uint32_t)(j >> 1) & 1u, abort_flag, p.spin_limit)) { ok = false; break; }
+          // the operands of both products that follow P(j) are waited for first (they arrive
+          // long before it), so that nothing stands between P(j) and S(j+2)
           if (!mbar_wait(v_full + j % VS, (uint32_t)(j / VS) & 1u, abort_flag, p.spin_limit)) { ok = false; break; }
+          if (j + 2 < T) wait_k(j + 2);
+          if (!ok) break;
+          if (!mbar_wait(p_ready + (j & 1), (uint32_t)(j >> 1) & 1u, abort_flag, p.spin_limit)) { ok = false; break; }
           tc_fence_after_sync();
           // O_w (+)= P[:, 64 w .. 64 w + 63] V[64 w .. 64 w + 63, :] for both warpgroups' halves
           const uint32_t a = tmem + kColS + (uint32_t)(j & 1) * BN;
@@ -389,7 +393,10 @@ graph_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
           umma_ts_k64(tmem + kColO + HD, a + 64u, vj + 4u * 128u, hi, idesc_o, j > 0 ? 1u : 0u);
           umma_commit(v_empty + j % VS);
           umma_commit(pv_done + (j & 1));
-          if (j + 2 < T) s_tile(j + 2);
+          if (j + 2 < T) {
+            issue_s(j + 2, j & 1, 0);
+            umma_commit(k_empty + (j + 2) % KS);
+          }
         }
       } else {
         // S buffer q belongs to M-tile q; a key tile serves both before it is released
