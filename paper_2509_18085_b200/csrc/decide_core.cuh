@@ -256,7 +256,7 @@ __device__ __forceinline__ bool finalize_row(const Partial* __restrict__ p, int 
     for (int u = 0; u < kBatch; ++u) {
       const int k = sub + kLanes * (t0 + u);
       q[u] = Partial{-INFINITY, 0.f, 0x7fffffff, 0};
-      if (k < splits) {  // read at L2: another grid wrote these while this CTA may already have been resident
+      if (k < splits && state == mask_id) {  // read at L2: another grid wrote these while this CTA may already have been resident; the slices of an unmasked row were never written
         const int4 w = __ldcg(reinterpret_cast<const int4*>(p + k));
         q[u] = Partial{__int_as_float(w.x), __int_as_float(w.y), w.z, w.w};
       }
