@@ -66,6 +66,15 @@ def test_draws_match_the_oracle(dtype, V, T):
         check(logits, tokens, mask, dtype, rule, S_, tau, T, seed=1234 + V)
 
 
+def test_more_slices_than_lanes_and_long_blocks():
+    """34 vocabulary slices (the slice choice loops over the lanes twice) and a
+    block of 40 positions (the masked count spans two ballots)."""
+    logits, tokens, mask = case(5, 1, 2, 3, 270000, "bf16", p_unmasked=0.0)
+    check(logits, tokens, mask, "bf16", spiffy.RULE_TOPS, 1, 0.0, 0.9, seed=31)
+    logits, tokens, mask = case(6, 1, 2, 40, 9000, "f32")
+    check(logits, tokens, mask, "f32", spiffy.RULE_THRESHOLD, 1, 0.05, 1.0, seed=32)
+
+
 def test_noise_ignores_the_node_and_follows_the_seed_and_the_state():
     logits, tokens, mask = case(3, 1, 1, 6, 5000, "f32", p_unmasked=0.0)
     x = np.repeat(logits, 4, axis=1)
