@@ -628,6 +628,12 @@ def main():
         for i in range(max(3, min(args.warmup, 2 * N_SETS))):
             step.run(sets[i % N_SETS])
         stream.synchronize()
+        # what the walk accepts on each input set: hops from the true block to the accepted node
+        accepted_depth = []
+        for x in sets:
+            step.run(x)
+            stream.synchronize()
+            accepted_depth += step.walk.n_accepted.tolist()
         before = spiffy.launch_count()
         graph = timer.capture([lambda x=x: step.run(x) for x in sets])
         launches_per_step = (spiffy.launch_count() - before) / N_SETS
@@ -780,6 +786,8 @@ def main():
                         "accept_walk": t_walk * 1e6, "decide_walk": t_dw * 1e6},
         "regions_ms_per_step": [r / N_SETS * 1e3 for r in regions],
         "dev_status": status,
+        "accepted_depth": {"per_input_set_and_sequence": accepted_depth,
+                           "histogram": {str(d): accepted_depth.count(d) for d in sorted(set(accepted_depth))}},
     }
     if composite is not None:
         line["composite_model_step"] = composite
